@@ -1,0 +1,224 @@
+/* mfet.h - C ABI of the multi-faceted embedding-table lookup library (sm_100a).
+ *
+ * The library computes the lookup path of a ranking model whose sparse ID
+ * features are embedded through large hashed tables:
+ *
+ *   raw 64-bit ID --hash--> table row --gather--> pooled (sum / mean / weighted
+ *   sum) over a ragged bag --> one dense fp32 row per sample, the outputs of all
+ *   (feature, table) slots side by side.
+ *
+ * Terms. A FEATURE is one ragged list of IDs per sample. A SLOT is one
+ * (feature, table) lookup that yields `dim` output columns; a multi-faceted
+ * feature has several slots, one per facet table, in adjacent columns. B is the
+ * batch size, F the number of features, L the number of slots, nnz the number
+ * of IDs in the batch.
+ *
+ * Conventions shared by every entry point.
+ *   - Return value: MFET_OK (0) or a negative MFET_ERR_* code. Nothing is
+ *     printed, thrown or aborted. Argument errors are found on the host before
+ *     anything is launched.
+ *   - "dev" pointers are device memory of the handle's GPU, "host" pointers are
+ *     ordinary host memory; the library never allocates device memory in any
+ *     call that takes a stream, and never frees or keeps ownership of caller
+ *     memory. Calls that take a stream are asynchronous on it and do not
+ *     synchronise, unless stated.
+ *   - `mfet_stream_t` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - No CPU fallback exists: every step runs in the library's own kernels.
+ */
+#ifndef MFET_H_
+#define MFET_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mfet_tables mfet_tables_t; /* opaque, library-owned */
+typedef void* mfet_stream_t;              /* a cudaStream_t */
+
+enum { MFET_F32 = 0, MFET_F16 = 1, MFET_BF16 = 2, MFET_INT4 = 3 };
+enum { MFET_POOL_SUM = 0, MFET_POOL_MEAN = 1, MFET_POOL_WSUM = 2 };
+enum { MFET_LOC_DEVICE = 0, MFET_LOC_HOST = 1 };
+enum { MFET_VAL_NORMAL = 0, MFET_VAL_GRID = 1 };
+
+enum {
+  MFET_OK = 0,
+  MFET_ERR_INVALID_ARG = -1,    /* null pointer, bad enum, bad size, bad id   */
+  MFET_ERR_NOT_REGISTERED = -2, /* host table used before its memory was given */
+  MFET_ERR_ALIGNMENT = -3,      /* pointer or stride not 16-byte aligned       */
+  MFET_ERR_UNSUPPORTED_DIM = -4,/* row bytes not a multiple of 16              */
+  MFET_ERR_WORKSPACE = -5,      /* workspace missing or too small              */
+  MFET_ERR_CUDA = -6,           /* a CUDA runtime call failed                  */
+  MFET_ERR_TIMEOUT = -7         /* reserved for bounded device-side waits      */
+};
+
+/* Bits of the device error word (mfet_query_status). */
+enum {
+  MFET_DEV_ROW_RANGE = 1u,      /* a pre-hashed row index was >= rows; skipped */
+  MFET_DEV_OFFSETS = 2u,        /* offsets decreased inside a bag; bag skipped */
+  MFET_DEV_CAPACITY = 4u        /* a host-path batch exceeded the workspace    */
+};
+
+/* One embedding table. Rows are `dim` elements of `dtype`, row-major.
+ * Paper, Section 2.2: categorical IDs reach their vectors through hashed
+ * lookup tables; `rows` is that table's vocabulary size. */
+typedef struct {
+  void* data;           /* MFET_LOC_DEVICE: dev pointer, 16-byte aligned, caller-owned,
+                           must outlive the handle. MFET_LOC_HOST: ignored (the memory
+                           is supplied later by mfet_host_tables_register).            */
+  uint64_t rows;        /* 1 .. 2^63-1                                                  */
+  uint32_t dim;         /* elements per row; stored row bytes must be a multiple of 16  */
+  uint32_t dtype;       /* MFET_F32 / MFET_F16 / MFET_BF16 / MFET_INT4                   */
+  uint32_t location;    /* MFET_LOC_DEVICE / MFET_LOC_HOST                              */
+  uint32_t flags;       /* must be 0                                                    */
+  uint64_t hash_seed;   /* XORed into the raw ID before hashing; 0 = plain hash         */
+  uint64_t row_stride_bytes; /* 0 = dense rows; otherwise >= row bytes, multiple of 16  */
+} mfet_table_desc_t;
+
+/* Shape of one batch. */
+typedef struct {
+  int32_t batch;               /* B >= 0                                              */
+  int32_t n_features;          /* F >= 1                                              */
+  int32_t n_slots;             /* L >= 1                                              */
+  int32_t flags;               /* bit0: `ids` already hold row indices (no hashing)   */
+  const int32_t* slot_feature; /* host int32[L]: feature read by each slot            */
+  int64_t out_ld;              /* floats per row of `out`; 0 = sum of the slots' dims */
+} mfet_batch_shape_t;
+
+/* Stored bytes of one row: dim*4 (F32), dim*2 (F16/BF16); INT4: dim/2 nibble
+ * bytes + fp16 scale + fp16 bias, rounded up to a multiple of 16 (dim even).
+ * Returns 0 for a bad dtype. */
+uint64_t mfet_row_bytes(uint32_t dim, uint32_t dtype);
+
+/* Create a table set on GPU `device` (a CUDA ordinal). Copies the descriptors;
+ * allocates only small host-side bookkeeping, one pinned status word, one
+ * internal stream and two events. Errors: INVALID_ARG (null, n_tables < 1, rows
+ * == 0, rows >= 2^63, bad dtype/location, flags != 0, null data for a device
+ * table), UNSUPPORTED_DIM, ALIGNMENT, CUDA. */
+int mfet_tables_create(const mfet_table_desc_t* descs /*host*/, int32_t n_tables, int32_t device,
+                       mfet_tables_t** out /*host*/);
+
+/* Destroy the handle; unpins only host memory that the library pinned itself.
+ * Synchronises the internal stream. NULL is accepted. */
+int mfet_tables_destroy(mfet_tables_t* t);
+
+/* Give a MFET_LOC_HOST table its memory (paper, Section 3.3: the largest tables
+ * stay in CPU memory while scoring runs on the GPU; here the GPU reads them in
+ * place through the unified address space instead of over an RPC).
+ * host_ptr: 16-byte-aligned host memory holding at least rows*stride bytes,
+ * caller-owned, valid until destroy. flags bit0 clear: the library pins and
+ * maps it (cudaHostRegister) and unpins it at destroy; bit0 set: the memory is
+ * already pinned and mapped. Errors: INVALID_ARG (bad id, not a host table,
+ * already registered, too few bytes), ALIGNMENT, CUDA. */
+int mfet_host_tables_register(mfet_tables_t* t, int32_t table_id, void* host_ptr, uint64_t bytes,
+                              uint32_t flags);
+
+/* rows_out[i] = splitmix64(ids[i] XOR hash_seed) mod rows of table `table_id`,
+ * as a non-negative int64 (paper, Section 2.2; the paper names no hash
+ * function, this is the library's). ids: dev u64[n]; rows_out: dev i64[n];
+ * n >= 0. In-place (rows_out aliasing ids) is allowed. */
+int mfet_hash_ids(const mfet_tables_t* t, int32_t table_id, const uint64_t* ids, int64_t n,
+                  int64_t* rows_out, mfet_stream_t stream);
+
+/* The lookup path for one batch (paper, Sections 1, 2.2, 3.3 and 4.1.1: hashed
+ * tables, several facet tables per ID feature all feeding the ranker, largest
+ * table in host memory). For slot s with feature f = slot_feature[s], table
+ * t = table_ids[s], D = dim_t, and sample b:
+ *   bag   = ids[offsets[f*B+b] .. offsets[f*B+b+1])
+ *   value = sum over the bag of c_i * row_t(hash_t(id_i)),  c_i = 1 (SUM, MEAN)
+ *           or weights[i] (WSUM); MEAN divides by the bag length; an empty bag
+ *           gives zeros
+ *   out[b*out_ld + col_s + d] = value[d],  col_s = sum of dims of slots before s.
+ * Accumulation is fp32 in an order that depends only on the inputs, so repeated
+ * calls give identical bits.
+ *   ids      dev u64[nnz], bags stored feature-major (all samples of feature 0,
+ *            then feature 1, ...)
+ *   offsets  dev i64[F*B + 1], nondecreasing
+ *   weights  dev f32[nnz], read only by WSUM slots; may be NULL if there is none
+ *   table_ids, pooling  host i32[L]
+ *   out      dev f32[B, out_ld]; the columns of all slots are fully overwritten
+ * Slots whose table is in host memory run on the library's internal stream
+ * (dedup -> cache probe -> host fetch -> pool), overlapped with the others and
+ * joined back into `stream`; they need a workspace (mfet_set_workspace) and
+ * `nnz_hint`-free operation: sizes are taken from the workspace capacity.
+ * Errors: INVALID_ARG, NOT_REGISTERED, WORKSPACE, CUDA. */
+int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape,
+                               const uint64_t* ids, const int64_t* offsets, const float* weights,
+                               const int32_t* table_ids, const int32_t* pooling, float* out,
+                               mfet_stream_t stream);
+
+/* In-batch dedup of hashed rows, done before host reads so that each distinct
+ * row crosses PCIe once (paper, Section 3.3 motivates keeping host traffic off
+ * the latency path). uniq = ascending distinct values of rows[0..n);
+ * inverse[i] = position of rows[i] in uniq; *n_unique = their number.
+ *   rows dev i64[n] (values in [0, 2^63)); uniq dev i64[n]; inverse dev i32[n];
+ *   n_unique dev i64[1]; 0 <= n <= workspace capacity.
+ * Uses the workspace. Errors: INVALID_ARG, WORKSPACE, CUDA. */
+int mfet_dedup_rows(mfet_tables_t* t, const int64_t* rows, int64_t n, int64_t* uniq,
+                    int32_t* inverse, int64_t* n_unique, mfet_stream_t stream);
+
+/* Device bytes that the hot-row cache of `n` rows of table `table_id` needs. */
+int mfet_cache_bytes(const mfet_tables_t* t, int32_t table_id, int64_t n, uint64_t* bytes /*host*/);
+
+/* Build the HBM cache of a host table (the paper leaves caching strategies as
+ * future work, Section 5; this is the library's): copies the listed rows from
+ * the registered host memory into `cache_mem` and builds the lookup index.
+ * rows_sorted: host i64[n], strictly increasing, each < rows. cache_mem: dev,
+ * 256-byte aligned, caller-owned, at least mfet_cache_bytes(); must stay valid
+ * while the handle uses it. n == 0 removes the cache. The call returns after
+ * the build has finished on `stream` (it synchronises that stream).
+ * Errors: INVALID_ARG, NOT_REGISTERED, ALIGNMENT, WORKSPACE (cache_bytes too small), CUDA. */
+int mfet_cache_build(mfet_tables_t* t, int32_t table_id, const int64_t* rows_sorted, int64_t n,
+                     void* cache_mem, uint64_t cache_bytes, mfet_stream_t stream);
+
+/* Workspace for the host-table path and mfet_dedup_rows: device bytes needed to
+ * handle up to `max_ids` IDs per host-table slot per call. */
+int mfet_workspace_bytes(const mfet_tables_t* t, int64_t max_ids, uint64_t* bytes /*host*/);
+
+/* Attach a caller-owned, 256-byte-aligned device workspace sized by
+ * mfet_workspace_bytes(max_ids). It must stay valid while the handle uses it;
+ * calls that use it must not overlap on the GPU. */
+int mfet_set_workspace(mfet_tables_t* t, void* dev_ptr, uint64_t bytes, int64_t max_ids);
+
+/* Same result as mfet_embedding_bag_forward with the batch in HOST memory: the
+ * call copies ids/offsets/weights to the device, runs the path, copies `out`
+ * back and waits for it. `dev_io` is caller-owned device scratch of at least
+ * mfet_host_io_bytes(); host buffers should be pinned for full copy speed.
+ * nnz = offsets[F*B]. */
+int mfet_host_io_bytes(const mfet_tables_t* t, const mfet_batch_shape_t* shape, const int32_t* table_ids,
+                       int64_t nnz, uint64_t* bytes /*host*/);
+int mfet_embedding_bag_forward_host(mfet_tables_t* t, const mfet_batch_shape_t* shape,
+                                    const uint64_t* ids_host, const int64_t* offsets_host,
+                                    const float* weights_host, int64_t nnz, const int32_t* table_ids,
+                                    const int32_t* pooling, float* out_host, void* dev_io,
+                                    uint64_t dev_io_bytes, mfet_stream_t stream);
+
+/* Synthetic table contents (the paper's tables are pretrained weights that are
+ * not public; this counter-based generator stands in for them):
+ *   k = r*dim + d;  u = splitmix64(value_key + k)
+ *   MFET_VAL_NORMAL: s = sum of the four 16-bit fields of u;
+ *                    v = float(s - 131070) * fp32(0.01 / 37837.227)
+ *   MFET_VAL_GRID:   v = float((u & 255) - 128) * 2^-13
+ * rounded to nearest-even into `dtype` (INT4: the row is then quantised: scale =
+ * fp16((max-min)/15), bias = fp16(min), code = clamp(rint((v-bias)/scale), 0, 15)).
+ * data: dev memory, or pinned+mapped host memory (written through the unified
+ * address space); rows [row0, row0+n_rows) are written. */
+int mfet_table_fill(void* data, uint64_t row0, uint64_t n_rows, uint32_t dim, uint32_t dtype,
+                    uint64_t row_stride_bytes, uint64_t value_key, uint32_t value_mode,
+                    mfet_stream_t stream);
+
+/* Read the device error word (bits MFET_DEV_*) without synchronising: it lives
+ * in pinned host memory that kernels write to. clear != 0 resets it. */
+int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits /*host*/, int32_t clear);
+
+/* Number of kernels the library has launched on behalf of this handle. */
+int mfet_launch_count(const mfet_tables_t* t, uint64_t* launches /*host*/);
+
+/* Static, human-readable name of a status code. */
+const char* mfet_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MFET_H_ */
