@@ -1,0 +1,441 @@
+#!/usr/bin/env python
+"""Benchmark of the embedding-table lookup path: pooled IDs per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+One step = one pass of the whole lookup path (hash -> gather -> pool -> concat, plus
+dedup -> cache probe -> host fetch for a host-resident table) over one synthetic batch.
+`value` is measured with the batch resident in HBM; `e2e` goes through the C-ABI call
+that takes HOST buffers (copies in and out inside the timed region). N > 1 runs N
+independent replicas (the path has no exchange step), one process per GPU.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2508_05700_b200 import inputs as gi  # noqa: E402
+
+METRIC = "pooled_ids_per_sec"
+UNIT = "IDs/s"
+DEFAULT_CONFIG = 3
+KERNEL_SOURCES = ["paper_2508_05700_b200/csrc/bag.cu", "paper_2508_05700_b200/csrc/common.cuh"]
+
+
+# ------------------------------------------------------------------ helpers --
+
+def algorithmic_bytes(w: gi.Workload, b: gi.Batch, slots=None) -> int:
+    """Bytes the method must move for one batch: one stored row per lookup, 8 per input ID
+    (+4 if weighted), 8 per bag offset, 4 per output element."""
+    B = w.batch
+    slots = range(w.n_slots) if slots is None else slots
+    feats = sorted({int(w.slot_feature[s]) for s in slots})
+    total = 0
+    out_dim = 0
+    for s in slots:
+        f = int(w.slot_feature[s])
+        t = w.tables[int(w.table_ids[s])]
+        n_f = int(b.offsets[(f + 1) * B] - b.offsets[f * B])
+        total += n_f * gi_row_bytes(t)
+        out_dim += t.dim
+    nnz = sum(int(b.offsets[(f + 1) * B] - b.offsets[f * B]) for f in feats)
+    total += nnz * (8 + (4 if b.weights is not None else 0))
+    total += (len(feats) * B + 1) * 8
+    total += B * out_dim * 4
+    return total
+
+
+def gi_row_bytes(t: gi.TableSpec) -> int:
+    return t.dim * (4 if t.dtype == gi.F32 else 2)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def kernel_fingerprint() -> str:
+    h = hashlib.sha256()
+    for p in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, p), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload_key: str):
+    """DRAM bytes per launch of the pooling kernel from the committed ncu summary; None when
+    there is none for this workload or the kernel sources changed since it was taken."""
+    path = os.path.join(ROOT, "profiles", "bag_kernel_dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    fp = kernel_fingerprint()
+    with open(path) as fh:
+        for line in fh:
+            if line.startswith("#") or not line.strip():
+                continue
+            key, fingerprint, nbytes = line.split()[:3]
+            if key == workload_key and fingerprint == fp:
+                return float(nbytes)
+    return None
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle sampling while the GPU is under load."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        for ts, line in self.lines:
+            if ts < t0 or ts > t1 + 0.15:
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax = float(f[2])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def aggregate_over_ranks(local_ms: float, local_units: float, dist=None):
+    """Slowest rank's time and the units all ranks processed (replicas: no data exchange)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return local_ms, local_units
+    import torch
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([local_ms], dtype=torch.float64, device=dev)
+    u = torch.tensor([local_units], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# --------------------------------------------------------------- CPU oracle --
+
+def oracle_tables(w: gi.Workload):
+    import oracle as orc
+    return [orc.Table(rows=s.rows, dim=s.dim, dtype=s.dtype, hash_seed=s.hash_seed, value_key=s.value_key)
+            for s in w.tables]
+
+
+def oracle_run_samples(w, b, tabs, samples, threads):
+    """The oracle, as it stands, over the given samples; sharded over samples on `threads`
+    host threads (the C routine runs without the interpreter lock)."""
+    import oracle as orc
+    chunks = [c for c in np.array_split(np.asarray(samples), threads) if c.size]
+
+    def run(c):
+        orc.embedding_bag(tabs, w.batch, w.n_features, w.slot_feature, w.table_ids, w.pooling, b.ids, b.offsets,
+                          b.weights, samples=c.tolist())
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=len(chunks)) as ex:
+        list(ex.map(run, chunks))
+    return time.perf_counter() - t0
+
+
+def ids_in_samples(w, b, samples):
+    off = b.offsets.reshape(-1)
+    n = 0
+    for f in range(w.n_features):
+        idx = f * w.batch + np.asarray(samples)
+        n += int((off[idx + 1] - off[idx]).sum())
+    return n
+
+
+def cpu_baseline(w, b, target_seconds=12.0):
+    import oracle as orc
+    orc.build()
+    tabs = oracle_tables(w)
+    threads = os.cpu_count() or 1
+    probe = list(range(min(w.batch, threads)))
+    dt = max(oracle_run_samples(w, b, tabs, probe, threads), 1e-4)
+    per_sample = dt / len(probe) * min(threads, len(probe)) / threads
+    n = int(min(w.batch, max(threads, target_seconds / max(per_sample, 1e-9))))
+    samples = list(range(n))
+    dt = oracle_run_samples(w, b, tabs, samples, threads)
+    n_ids = ids_in_samples(w, b, samples)
+    return {"value": n_ids / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "samples 0..%d of batch 0 (%d IDs) of %s, procedural table values, %.1f s" % (n - 1, n_ids, w.name, dt)}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on this machine's host cores, each step a bounded
+    sample of the workload."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    import oracle as orc
+    orc.build()
+    w = gi.make_workload(args.config)
+    b = gi.make_batch(w, 0)
+    tabs = oracle_tables(w)
+    threads = os.cpu_count() or 1
+    probe = list(range(min(w.batch, threads)))
+    dt = max(oracle_run_samples(w, b, tabs, probe, threads), 1e-4)
+    budget = 90.0 / max(1, args.steps + args.warmup)
+    n = int(min(w.batch, max(threads, budget / (dt / len(probe)))))
+    times, ids_done = [], 0
+    for step in range(args.warmup + args.steps):
+        lo = (step * n) % max(1, w.batch - n + 1)
+        samples = list(range(lo, lo + n))
+        dt = oracle_run_samples(w, b, tabs, samples, threads)
+        if step >= args.warmup:
+            times.append(dt)
+            ids_done += ids_in_samples(w, b, samples)
+    total = sum(times)
+    value = ids_done / total
+    sample = "%d samples of batch 0 per step (%d IDs per step on average), procedural table values" % (
+        n, ids_done // max(1, args.steps))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(1, args.steps),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "config": args.config},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------ GPU arm --
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2508_05700_b200 import build as b_
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    else:
+        torch.cuda.set_device(0)
+    if rank == 0:
+        b_.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2508_05700_b200 import mfet as m
+    from paper_2508_05700_b200.runtime import LookupEngine
+
+    w = gi.make_workload(args.config, rows_scale=args.rows_scale)
+    n_rot = args.batches
+    batches = [gi.make_batch(w, rank * 1000 + j) for j in range(n_rot)]
+    base = cpu_baseline(w, batches[0]) if (rank == 0 and world == 1 and not args.no_cpu_baseline) else None
+
+    dev = torch.cuda.current_device()
+    eng = LookupEngine(w, device=dev)
+    stream = torch.cuda.current_stream()
+    host_tabs = eng.host_table_ids()
+    cached_rows = 0
+    if host_tabs:
+        B = w.batch
+        host_feats = {int(w.slot_feature[s]) for s in range(w.n_slots) if int(w.table_ids[s]) in host_tabs}
+        worst = max(int(b.offsets[(f + 1) * B] - b.offsets[f * B]) for b in batches for f in host_feats)
+        eng.set_workspace(int(worst * 1.25) + 4096)
+        for t in host_tabs:
+            f = int(w.slot_feature[list(w.table_ids).index(t)])
+            cached_rows = eng.build_hot_cache(t, f, int(w.tables[t].rows * w.cache_fraction))
+
+    d_ids = [torch.from_numpy(b.ids.view(np.int64)).cuda() for b in batches]
+    d_off = [torch.from_numpy(b.offsets).cuda() for b in batches]
+    d_w = [None if b.weights is None else torch.from_numpy(b.weights).cuda() for b in batches]
+    out = torch.empty(w.batch, w.out_dim, dtype=torch.float32, device="cuda")
+    nnz = [int(b.offsets[-1]) for b in batches]
+
+    def step(j):
+        k = j % n_rot
+        eng.forward(d_ids[k], d_off[k], d_w[k], out)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(dev)
+    if rank == 0:
+        sampler.start()
+    # warm-up: W steps, then keep the GPU under the same load for about a second so that the
+    # clock samples around the timed region describe the loaded state
+    for j in range(args.warmup):
+        step(j)
+    torch.cuda.synchronize()
+    t_load0 = time.time()
+    j = args.warmup
+    while time.time() - t_load0 < args.load_seconds:
+        for _ in range(50):
+            step(j)
+            j += 1
+        torch.cuda.synchronize()
+
+    # ---- timed region: exactly K steps, inputs resident in HBM ----------------
+    launches0 = m.mfet_launch_count(eng.h)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for j in range(args.steps):
+        step(j)
+    e1.record(stream)
+    barrier()
+    local_ms = e0.elapsed_time(e1)
+    launches = m.mfet_launch_count(eng.h) - launches0
+    ids_done = sum(nnz[j % n_rot] for j in range(args.steps))
+    assert m.mfet_query_status(eng.h) == 0, "device error bits set during the timed region"
+
+    # ---- dominant kernel alone: the pooling kernel over the HBM-resident slots --
+    dev_slots = [s for s in range(w.n_slots) if w.tables[int(w.table_ids[s])].location == gi.LOC_DEVICE]
+    if len(dev_slots) == w.n_slots:
+        kern_ms = local_ms / args.steps
+    else:
+        sub_shape, keep = m.make_shape(w.batch, w.n_features, w.slot_feature[dev_slots])
+        sub_out = torch.empty(w.batch, sum(w.tables[int(w.table_ids[s])].dim for s in dev_slots), device="cuda")
+        k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for rep in range(2):
+            k0.record(stream)
+            for j in range(args.steps):
+                k = j % n_rot
+                eng.forward(d_ids[k], d_off[k], d_w[k], sub_out, table_ids=w.table_ids[dev_slots],
+                            pooling=w.pooling[dev_slots], shape=sub_shape)
+            k1.record(stream)
+            torch.cuda.synchronize()
+        kern_ms = k0.elapsed_time(k1) / args.steps
+    alg = float(np.mean([algorithmic_bytes(w, batches[j % n_rot], dev_slots) for j in range(min(args.steps, n_rot))]))
+
+    # ---- end to end: host buffers in, host result out, through the C-ABI call ---
+    p_ids = [torch.from_numpy(b.ids.view(np.int64)).pin_memory() for b in batches]
+    p_off = [torch.from_numpy(b.offsets).pin_memory() for b in batches]
+    p_w = [None if b.weights is None else torch.from_numpy(b.weights).pin_memory() for b in batches]
+    p_out = torch.empty(w.batch, w.out_dim, dtype=torch.float32).pin_memory()
+    io_bytes = max(m.mfet_host_io_bytes(eng.h, eng.shape, w.table_ids, n) for n in nnz)
+    io = torch.empty(io_bytes, dtype=torch.uint8, device="cuda")
+
+    def e2e_step(j):
+        k = j % n_rot
+        m.mfet_embedding_bag_forward_host(eng.h, eng.shape, p_ids[k], p_off[k], p_w[k], nnz[k], w.table_ids,
+                                          w.pooling, p_out, io, io_bytes, eng.stream)
+    for j in range(max(3, args.warmup)):
+        e2e_step(j)
+    barrier()
+    e0.record(stream)
+    for j in range(args.steps):
+        e2e_step(j)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    t_load1 = time.time()
+    clocks = sampler.stop(t_load0, t_load1) if rank == 0 else None
+
+    h2d = float(np.mean([nnz[k] * (8 + (4 if batches[k].weights is not None else 0)) + batches[k].offsets.size * 8
+                         for k in range(n_rot)]))
+    d2h = float(w.batch * w.out_dim * 4)
+
+    ms, units = aggregate_over_ranks(local_ms, float(ids_done), dist if world > 1 else None)
+    e2e_ms_all, _ = aggregate_over_ranks(e2e_ms, float(ids_done), dist if world > 1 else None)
+    eng.close()
+    if world > 1:
+        dist.destroy_process_group()
+    if rank != 0:
+        return 0
+
+    peak, peak_kind = measured_peaks()
+    achieved = alg / (kern_ms * 1e-3) / 1e9
+    wl_key = "config%d" % args.config + ("" if args.rows_scale == 1.0 else "_rows%g" % args.rows_scale)
+    line = {
+        "metric": METRIC, "value": units / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "config": args.config, "batch": w.batch, "ids_per_step": float(np.mean(nnz)),
+                   "row_lookups_per_step": float(np.mean([sum(int(b.offsets[(int(w.slot_feature[s]) + 1) * w.batch] -
+                                                                   b.offsets[int(w.slot_feature[s]) * w.batch])
+                                                               for s in range(w.n_slots)) for b in batches])),
+                   "table_bytes": int(sum(t.rows * gi_row_bytes(t) for t in w.tables)),
+                   "rows_scale": args.rows_scale, "cached_rows": cached_rows,
+                   "l2": "no flush: tables are far larger than L2 and %d distinct batches rotate" % n_rot,
+                   "parallelism": "replicas x%d" % world},
+        "e2e": {"value": units / (e2e_ms_all * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": recorded_traffic(wl_key), "peak_kind": peak_kind + " copy bandwidth",
+                     "kernel": "bag_kernel (all HBM-resident slots, one launch)",
+                     "algorithmic_bytes_per_launch": alg, "kernel_ms": kern_ms},
+        "cpu_baseline": base,
+        "clocks": clocks,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--impl", default="mfet", choices=["mfet", "reference"])
+    ap.add_argument("--rows-scale", type=float, default=1.0, help="shrink table rows (reported in config)")
+    ap.add_argument("--batches", type=int, default=8, help="distinct batches rotated through")
+    ap.add_argument("--load-seconds", type=float, default=1.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

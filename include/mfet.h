@@ -34,6 +34,12 @@
 extern "C" {
 #endif
 
+#if defined(__GNUC__)
+#define MFET_API __attribute__((visibility("default")))
+#else
+#define MFET_API
+#endif
+
 typedef struct mfet_tables mfet_tables_t; /* opaque, library-owned */
 typedef void* mfet_stream_t;              /* a cudaStream_t */
 
@@ -41,6 +47,7 @@ enum { MFET_F32 = 0, MFET_F16 = 1, MFET_BF16 = 2, MFET_INT4 = 3 };
 enum { MFET_POOL_SUM = 0, MFET_POOL_MEAN = 1, MFET_POOL_WSUM = 2 };
 enum { MFET_LOC_DEVICE = 0, MFET_LOC_HOST = 1 };
 enum { MFET_VAL_NORMAL = 0, MFET_VAL_GRID = 1 };
+enum { MFET_OPT_GROUP_POLICY = 1 };
 
 enum {
   MFET_OK = 0,
@@ -89,19 +96,19 @@ typedef struct {
 /* Stored bytes of one row: dim*4 (F32), dim*2 (F16/BF16); INT4: dim/2 nibble
  * bytes + fp16 scale + fp16 bias, rounded up to a multiple of 16 (dim even).
  * Returns 0 for a bad dtype. */
-uint64_t mfet_row_bytes(uint32_t dim, uint32_t dtype);
+MFET_API uint64_t mfet_row_bytes(uint32_t dim, uint32_t dtype);
 
 /* Create a table set on GPU `device` (a CUDA ordinal). Copies the descriptors;
  * allocates only small host-side bookkeeping, one pinned status word, one
  * internal stream and two events. Errors: INVALID_ARG (null, n_tables < 1, rows
  * == 0, rows >= 2^63, bad dtype/location, flags != 0, null data for a device
  * table), UNSUPPORTED_DIM, ALIGNMENT, CUDA. */
-int mfet_tables_create(const mfet_table_desc_t* descs /*host*/, int32_t n_tables, int32_t device,
+MFET_API int mfet_tables_create(const mfet_table_desc_t* descs /*host*/, int32_t n_tables, int32_t device,
                        mfet_tables_t** out /*host*/);
 
 /* Destroy the handle; unpins only host memory that the library pinned itself.
  * Synchronises the internal stream. NULL is accepted. */
-int mfet_tables_destroy(mfet_tables_t* t);
+MFET_API int mfet_tables_destroy(mfet_tables_t* t);
 
 /* Give a MFET_LOC_HOST table its memory (paper, Section 3.3: the largest tables
  * stay in CPU memory while scoring runs on the GPU; here the GPU reads them in
@@ -111,14 +118,14 @@ int mfet_tables_destroy(mfet_tables_t* t);
  * maps it (cudaHostRegister) and unpins it at destroy; bit0 set: the memory is
  * already pinned and mapped. Errors: INVALID_ARG (bad id, not a host table,
  * already registered, too few bytes), ALIGNMENT, CUDA. */
-int mfet_host_tables_register(mfet_tables_t* t, int32_t table_id, void* host_ptr, uint64_t bytes,
+MFET_API int mfet_host_tables_register(mfet_tables_t* t, int32_t table_id, void* host_ptr, uint64_t bytes,
                               uint32_t flags);
 
 /* rows_out[i] = splitmix64(ids[i] XOR hash_seed) mod rows of table `table_id`,
  * as a non-negative int64 (paper, Section 2.2; the paper names no hash
  * function, this is the library's). ids: dev u64[n]; rows_out: dev i64[n];
  * n >= 0. In-place (rows_out aliasing ids) is allowed. */
-int mfet_hash_ids(const mfet_tables_t* t, int32_t table_id, const uint64_t* ids, int64_t n,
+MFET_API int mfet_hash_ids(const mfet_tables_t* t, int32_t table_id, const uint64_t* ids, int64_t n,
                   int64_t* rows_out, mfet_stream_t stream);
 
 /* The lookup path for one batch (paper, Sections 1, 2.2, 3.3 and 4.1.1: hashed
@@ -133,7 +140,7 @@ int mfet_hash_ids(const mfet_tables_t* t, int32_t table_id, const uint64_t* ids,
  * Accumulation is fp32 in an order that depends only on the inputs, so repeated
  * calls give identical bits.
  *   ids      dev u64[nnz], bags stored feature-major (all samples of feature 0,
- *            then feature 1, ...)
+ *            then feature 1, ...); never NULL, even when nnz == 0
  *   offsets  dev i64[F*B + 1], nondecreasing
  *   weights  dev f32[nnz], read only by WSUM slots; may be NULL if there is none
  *   table_ids, pooling  host i32[L]
@@ -143,7 +150,7 @@ int mfet_hash_ids(const mfet_tables_t* t, int32_t table_id, const uint64_t* ids,
  * joined back into `stream`; they need a workspace (mfet_set_workspace) and
  * `nnz_hint`-free operation: sizes are taken from the workspace capacity.
  * Errors: INVALID_ARG, NOT_REGISTERED, WORKSPACE, CUDA. */
-int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape,
+MFET_API int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape,
                                const uint64_t* ids, const int64_t* offsets, const float* weights,
                                const int32_t* table_ids, const int32_t* pooling, float* out,
                                mfet_stream_t stream);
@@ -153,13 +160,15 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
  * the latency path). uniq = ascending distinct values of rows[0..n);
  * inverse[i] = position of rows[i] in uniq; *n_unique = their number.
  *   rows dev i64[n] (values in [0, 2^63)); uniq dev i64[n]; inverse dev i32[n];
- *   n_unique dev i64[1]; 0 <= n <= workspace capacity.
+ *   n_unique dev i64[1]; 0 <= n <= workspace capacity (and n < 2^31).
+ *   max_row: exclusive upper bound of the values if known (it shortens the
+ *   sort), 0 if unknown. A value >= max_row gives an undefined order.
  * Uses the workspace. Errors: INVALID_ARG, WORKSPACE, CUDA. */
-int mfet_dedup_rows(mfet_tables_t* t, const int64_t* rows, int64_t n, int64_t* uniq,
-                    int32_t* inverse, int64_t* n_unique, mfet_stream_t stream);
+MFET_API int mfet_dedup_rows(mfet_tables_t* t, const int64_t* rows, int64_t n, int64_t* uniq,
+                    int32_t* inverse, int64_t* n_unique, int64_t max_row, mfet_stream_t stream);
 
 /* Device bytes that the hot-row cache of `n` rows of table `table_id` needs. */
-int mfet_cache_bytes(const mfet_tables_t* t, int32_t table_id, int64_t n, uint64_t* bytes /*host*/);
+MFET_API int mfet_cache_bytes(const mfet_tables_t* t, int32_t table_id, int64_t n, uint64_t* bytes /*host*/);
 
 /* Build the HBM cache of a host table (the paper leaves caching strategies as
  * future work, Section 5; this is the library's): copies the listed rows from
@@ -169,26 +178,26 @@ int mfet_cache_bytes(const mfet_tables_t* t, int32_t table_id, int64_t n, uint64
  * while the handle uses it. n == 0 removes the cache. The call returns after
  * the build has finished on `stream` (it synchronises that stream).
  * Errors: INVALID_ARG, NOT_REGISTERED, ALIGNMENT, WORKSPACE (cache_bytes too small), CUDA. */
-int mfet_cache_build(mfet_tables_t* t, int32_t table_id, const int64_t* rows_sorted, int64_t n,
+MFET_API int mfet_cache_build(mfet_tables_t* t, int32_t table_id, const int64_t* rows_sorted, int64_t n,
                      void* cache_mem, uint64_t cache_bytes, mfet_stream_t stream);
 
 /* Workspace for the host-table path and mfet_dedup_rows: device bytes needed to
  * handle up to `max_ids` IDs per host-table slot per call. */
-int mfet_workspace_bytes(const mfet_tables_t* t, int64_t max_ids, uint64_t* bytes /*host*/);
+MFET_API int mfet_workspace_bytes(const mfet_tables_t* t, int64_t max_ids, uint64_t* bytes /*host*/);
 
 /* Attach a caller-owned, 256-byte-aligned device workspace sized by
  * mfet_workspace_bytes(max_ids). It must stay valid while the handle uses it;
  * calls that use it must not overlap on the GPU. */
-int mfet_set_workspace(mfet_tables_t* t, void* dev_ptr, uint64_t bytes, int64_t max_ids);
+MFET_API int mfet_set_workspace(mfet_tables_t* t, void* dev_ptr, uint64_t bytes, int64_t max_ids);
 
 /* Same result as mfet_embedding_bag_forward with the batch in HOST memory: the
  * call copies ids/offsets/weights to the device, runs the path, copies `out`
  * back and waits for it. `dev_io` is caller-owned device scratch of at least
  * mfet_host_io_bytes(); host buffers should be pinned for full copy speed.
  * nnz = offsets[F*B]. */
-int mfet_host_io_bytes(const mfet_tables_t* t, const mfet_batch_shape_t* shape, const int32_t* table_ids,
+MFET_API int mfet_host_io_bytes(const mfet_tables_t* t, const mfet_batch_shape_t* shape, const int32_t* table_ids,
                        int64_t nnz, uint64_t* bytes /*host*/);
-int mfet_embedding_bag_forward_host(mfet_tables_t* t, const mfet_batch_shape_t* shape,
+MFET_API int mfet_embedding_bag_forward_host(mfet_tables_t* t, const mfet_batch_shape_t* shape,
                                     const uint64_t* ids_host, const int64_t* offsets_host,
                                     const float* weights_host, int64_t nnz, const int32_t* table_ids,
                                     const int32_t* pooling, float* out_host, void* dev_io,
@@ -204,19 +213,25 @@ int mfet_embedding_bag_forward_host(mfet_tables_t* t, const mfet_batch_shape_t* 
  * fp16((max-min)/15), bias = fp16(min), code = clamp(rint((v-bias)/scale), 0, 15)).
  * data: dev memory, or pinned+mapped host memory (written through the unified
  * address space); rows [row0, row0+n_rows) are written. */
-int mfet_table_fill(void* data, uint64_t row0, uint64_t n_rows, uint32_t dim, uint32_t dtype,
+MFET_API int mfet_table_fill(void* data, uint64_t row0, uint64_t n_rows, uint32_t dim, uint32_t dtype,
                     uint64_t row_stride_bytes, uint64_t value_key, uint32_t value_mode,
                     mfet_stream_t stream);
 
 /* Read the device error word (bits MFET_DEV_*) without synchronising: it lives
  * in pinned host memory that kernels write to. clear != 0 resets it. */
-int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits /*host*/, int32_t clear);
+MFET_API int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits /*host*/, int32_t clear);
+
+/* Tuning knobs. MFET_OPT_GROUP_POLICY: how the pooling kernel maps lanes to
+ * bags: 0 = chosen per tile from its mean bag length (default), 1 = one row
+ * group per bag (best for short bags), 2 = one warp per bag (long bags). The
+ * result is the same up to the order of fp32 additions. */
+MFET_API int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value);
 
 /* Number of kernels the library has launched on behalf of this handle. */
-int mfet_launch_count(const mfet_tables_t* t, uint64_t* launches /*host*/);
+MFET_API int mfet_launch_count(const mfet_tables_t* t, uint64_t* launches /*host*/);
 
 /* Static, human-readable name of a status code. */
-const char* mfet_status_string(int status);
+MFET_API const char* mfet_status_string(int status);
 
 #ifdef __cplusplus
 }

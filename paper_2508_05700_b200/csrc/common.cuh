@@ -1,0 +1,216 @@
+// Shared declarations of the mfet library: handle layout, kernel parameter
+// blocks, and the small device helpers (hash, exact modulo, cache-hinted
+// loads/stores) that several kernels use.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/mfet.h"
+
+namespace mfet {
+
+// ------------------------------------------------------------ host side -----
+
+struct CacheInfo {
+  const int64_t* keys = nullptr;         // dev i64[n], ascending
+  const uint32_t* bucket_start = nullptr;// dev u32[n_buckets + 1]
+  const uint8_t* data = nullptr;         // dev [n, row_bytes]
+  int64_t n = 0;
+  uint32_t bucket_shift = 0;             // bucket = key >> bucket_shift
+  uint32_t n_buckets = 0;
+};
+
+struct TableHost {
+  mfet_table_desc_t desc;
+  uint64_t row_bytes = 0;
+  uint64_t stride = 0;
+  uint64_t magic = 0;        // floor((2^64 - 1) / rows)
+  const uint8_t* dev_ptr = nullptr;  // device-visible address of the rows
+  void* host_ptr = nullptr;
+  bool registered = false;   // host table: memory supplied
+  bool pinned_by_us = false;
+  CacheInfo cache;
+};
+
+}  // namespace mfet
+
+struct mfet_tables {
+  int device = 0;
+  std::vector<mfet::TableHost> tables;
+  uint32_t* err_host = nullptr;  // pinned + mapped status word
+  uint32_t* err_dev = nullptr;   // its device-visible address
+  cudaStream_t side = nullptr;   // host-table slots run here
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  void* ws = nullptr;
+  uint64_t ws_bytes = 0;
+  int64_t ws_max_ids = 0;
+  uint64_t launches = 0;
+  int32_t group_policy = 0;
+};
+
+namespace mfet {
+
+// ----------------------------------------------------------- kernel params --
+
+// One (feature, table) slot as the pooling kernel sees it. Rows wider than 512
+// bytes are split on the host into several entries of at most 32 chunks.
+struct SlotDev {
+  const uint8_t* table;  // first byte of the slot's column block in row 0
+  uint64_t rows;
+  uint64_t magic;
+  uint64_t seed;
+  uint64_t stride;       // bytes between rows
+  uint32_t feature;
+  uint32_t col_off;      // first output column
+  uint16_t chunks;       // 16-byte chunks of the row that this entry covers (1..32)
+  uint8_t dtype;
+  uint8_t pooling;
+  uint8_t lpr_log2;      // lanes per row = 1 << lpr_log2 >= chunks
+  uint8_t narrow;        // 1: (rows*stride)/16 fits 32 bits
+  uint16_t pad;
+  uint32_t pad2;
+};
+static_assert(sizeof(SlotDev) == 64, "SlotDev must stay 64 bytes");
+
+constexpr int kMaxSlotsPerLaunch = 56;
+constexpr int kMaxTile = 64;
+
+struct BagParams {
+  const uint64_t* ids;
+  const int64_t* offsets;
+  const float* weights;
+  float* out;
+  uint32_t* err;
+  int64_t out_ld;
+  int32_t batch;
+  int32_t n_slots;
+  int32_t tiles_per_slot;
+  int32_t tile;          // bags per block, <= kMaxTile
+  uint32_t flags;        // bit0: ids are rows; bit1: out allows 16-byte vector stores
+  int32_t group_policy;  // 0 auto, 1 one row-group per bag, 2 one warp per bag
+  SlotDev slot[kMaxSlotsPerLaunch];
+};
+static_assert(sizeof(BagParams) <= 4000, "BagParams must fit the kernel parameter space");
+
+// ---------------------------------------------------------- device helpers --
+
+// splitmix64 output function (public domain; Steele, Lea, Flood).
+__host__ __device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
+  x += 0x9E3779B97F4A7C15ULL;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ULL;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBULL;
+  return x ^ (x >> 31);
+}
+
+// Exact h mod d for a runtime divisor, with magic = floor((2^64-1)/d).
+// q = floor(h*magic / 2^64) underestimates floor(h/d) by at most 2, so the
+// remainder estimate is below 3d and two conditional subtractions finish it.
+__device__ __forceinline__ uint64_t mod_rows(uint64_t h, uint64_t d, uint64_t magic) {
+  uint64_t q = __umul64hi(h, magic);
+  uint64_t r = h - q * d;
+  if (r >= d) r -= d;
+  if (r >= d) r -= d;
+  return r;
+}
+
+inline uint64_t host_magic(uint64_t rows) { return 0xFFFFFFFFFFFFFFFFULL / rows; }
+
+// 16-byte row load that stays out of L1 (rows are reused across SMs through
+// L2 only) through the read-only path.
+__device__ __forceinline__ uint4 ld_row16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ float bf16lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t x) { return __uint_as_float(x & 0xFFFF0000u); }
+
+// ------------------------------------------------- host-table path params --
+
+// Element count of a pass: immediate, or the ID count of one feature read from
+// the CSR offsets on the device (the host never learns it).
+struct NSrc {
+  const int64_t* offsets;  // nullptr => n_imm
+  int64_t idx_lo, idx_hi;  // n = offsets[idx_hi] - offsets[idx_lo]
+  int64_t n_imm;
+  int64_t cap;             // counts above cap (or negative) degrade to 0
+};
+
+struct CacheDev {
+  const int64_t* keys;
+  const uint32_t* bucket_start;
+  const uint8_t* data;
+  int64_t n;
+  uint32_t bucket_shift;
+  uint32_t pad;
+};
+
+struct WsLayout {
+  uint64_t keys_a, keys_b, idx_a, idx_b, hist, tile_counts, counters, uniq, inverse, src, miss_rows,
+      staging, total;
+  int nblk_sort, nblk_scan;
+};
+
+struct HashArgs {
+  const uint64_t* ids;
+  uint64_t seed, rows, magic;
+  uint32_t pre_hashed;
+};
+
+struct DedupArgs {
+  NSrc ns;
+  const uint64_t* first_keys;  // pass-0 input when hash == nullptr
+  const HashArgs* hash;        // non-null: pass 0 hashes the slot's raw IDs
+  uint64_t max_key;            // largest possible key (sets the number of passes)
+  void* ws;
+  WsLayout layout;
+  const CacheDev* cache;       // non-null: probe + miss compaction
+  int64_t* uniq;
+  int32_t* inverse;
+  int64_t* n_unique;
+  int32_t* src;
+  int64_t* miss_rows;
+  int64_t* n_miss;
+  uint32_t* err;
+};
+
+// Where the pooling kernel finds the rows of a host-table slot.
+struct IndirectParams {
+  const int32_t* inverse;     // [n] position in uniq of every lookup of the slot
+  const int32_t* src;         // [n_unique] >= 0: cache slot; < 0: -1 - staging index
+  const uint8_t* cache_data;
+  const uint8_t* staging;
+  uint64_t row_bytes;
+  int64_t cap;
+};
+
+struct CacheLayout {
+  uint64_t keys, bucket_start, data, total;
+  uint32_t bucket_shift, n_buckets;
+};
+
+uint64_t workspace_layout(int64_t max_ids, uint64_t max_row_bytes, WsLayout* L);
+void cache_layout(uint64_t rows, int64_t n, uint64_t row_bytes, CacheLayout* L);
+cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s);
+cudaError_t launch_fetch(const uint8_t* table, uint64_t stride, uint32_t chunks, const int64_t* rows_list,
+                         const int64_t* n_ptr, int64_t n_imm, uint8_t* dst, cudaStream_t s);
+cudaError_t launch_bag_indirect(const BagParams& p, const IndirectParams& ip, cudaStream_t s);
+int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, int32_t feature, int32_t pooling,
+                  uint32_t col, cudaStream_t side);
+
+// launch helpers implemented in the kernel files
+cudaError_t launch_hash(const uint64_t* ids, int64_t n, uint64_t seed, uint64_t rows, uint64_t magic,
+                        int64_t* rows_out, cudaStream_t s);
+cudaError_t launch_fill(void* data, uint64_t row0, uint64_t n_rows, uint32_t dim, uint32_t dtype,
+                        uint64_t stride, uint64_t key, uint32_t mode, cudaStream_t s);
+cudaError_t launch_bag(const BagParams& p, cudaStream_t s);
+
+}  // namespace mfet

@@ -1,0 +1,444 @@
+// K-dedup: in-batch dedup of hashed rows = stable LSD radix sort of (row, index)
+// pairs, then adjacent-unique with an inverse map. For a host-table slot the
+// same pass also probes the HBM hot-row cache and compacts the misses, so that
+// only distinct, uncached rows are fetched over PCIe.
+//
+// Every kernel here is a plain data-parallel pass; the passes are ordered by the
+// stream, so no kernel ever waits on another block. Results are canonical
+// (ascending unique rows), hence bit-reproducible.
+#include "common.cuh"
+
+namespace mfet {
+
+namespace {
+
+constexpr int kSortThreads = 256;
+constexpr int kSortRounds = 8;
+constexpr int kSortTile = kSortThreads * kSortRounds;  // keys per block per pass
+constexpr int kScanThreads = 256;
+constexpr int kScanItems = 4;
+constexpr int kScanTile = kScanThreads * kScanItems;
+
+// Number of elements: either immediate, or the ID count of feature f taken
+// from the CSR offsets on the device. Out-of-capacity or negative counts
+// degrade to 0 (the caller flags MFET_DEV_CAPACITY once).
+__device__ __forceinline__ int64_t resolve_n(const NSrc& s, int64_t* lo) {
+  if (s.offsets == nullptr) {
+    *lo = 0;
+    return s.n_imm;
+  }
+  const int64_t a = s.offsets[s.idx_lo], b = s.offsets[s.idx_hi];
+  *lo = a;
+  const int64_t n = b - a;
+  return (n < 0 || n > s.cap) ? 0 : n;
+}
+
+// ---- pass kernels --------------------------------------------------------
+
+// Digit histogram of one tile. With HASH the keys are produced here from the
+// raw IDs (first pass of a host-table slot) and stored for the later passes.
+template <bool HASH>
+__global__ void __launch_bounds__(kSortThreads) hist_kernel(NSrc ns, const uint64_t* __restrict__ keys_in,
+                                                            uint64_t* __restrict__ keys_store,
+                                                            const uint64_t* __restrict__ ids, uint64_t seed,
+                                                            uint64_t rows, uint64_t magic, uint32_t pre_hashed,
+                                                            int shift, uint32_t* __restrict__ hist, int nblk,
+                                                            uint32_t* err) {
+  __shared__ uint32_t h[256];
+  int64_t lo;
+  const int64_t n = resolve_n(ns, &lo);
+  if (HASH && blockIdx.x == 0 && threadIdx.x == 0 && ns.offsets) {
+    const int64_t raw = ns.offsets[ns.idx_hi] - ns.offsets[ns.idx_lo];
+    if (raw < 0) atomicOr(err, (uint32_t)MFET_DEV_OFFSETS);
+    if (raw > ns.cap) atomicOr(err, (uint32_t)MFET_DEV_CAPACITY);
+  }
+  h[threadIdx.x] = 0;
+  __syncthreads();
+  const int64_t base = (int64_t)blockIdx.x * kSortTile;
+#pragma unroll
+  for (int r = 0; r < kSortRounds; ++r) {
+    const int64_t i = base + r * kSortThreads + threadIdx.x;
+    if (i < n) {
+      uint64_t k;
+      if (HASH) {
+        const uint64_t id = __ldcs(reinterpret_cast<const unsigned long long*>(ids) + lo + i);
+        k = pre_hashed ? id : mod_rows(splitmix64(id ^ seed), rows, magic);
+        if (k >= rows) {  // only possible for pre-hashed input
+          atomicOr(err, (uint32_t)MFET_DEV_ROW_RANGE);
+          k = rows - 1;
+        }
+        keys_store[i] = k;
+      } else {
+        k = keys_in[i];
+      }
+      atomicAdd(&h[(k >> shift) & 255u], 1u);
+    }
+  }
+  __syncthreads();
+  hist[(size_t)threadIdx.x * nblk + blockIdx.x] = h[threadIdx.x];
+}
+
+// Exclusive scan of `total` counters in place, one block. Each thread owns a
+// contiguous segment; segment sums are scanned with shuffles.
+__global__ void __launch_bounds__(1024) scan_counters_kernel(uint32_t* __restrict__ a, int total) {
+  __shared__ uint32_t warp_sum[32];
+  const int per = (total + 1023) / 1024;
+  const int begin = min(total, (int)threadIdx.x * per), end = min(total, begin + per);
+  uint32_t sum = 0;
+  for (int i = begin; i < end; ++i) sum += a[i];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = sum;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+    if (lane >= d) inc += t;
+  }
+  if (lane == 31) warp_sum[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = warp_sum[lane];
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, w, d);
+      if (lane >= d) w += t;
+    }
+    warp_sum[lane] = w;
+  }
+  __syncthreads();
+  uint32_t run = inc - sum + (warp ? warp_sum[warp - 1] : 0u);
+  for (int i = begin; i < end; ++i) {
+    const uint32_t v = a[i];
+    a[i] = run;
+    run += v;
+  }
+}
+
+// Stable scatter of one tile by the current digit. Rounds of 256 keys keep the
+// input order: within a round, warps are ordered through per-warp digit counts
+// and lanes through match_any masks.
+__global__ void __launch_bounds__(kSortThreads) scatter_kernel(NSrc ns, const uint64_t* __restrict__ keys_in,
+                                                               const uint32_t* __restrict__ idx_in,
+                                                               uint64_t* __restrict__ keys_out,
+                                                               uint32_t* __restrict__ idx_out, int shift,
+                                                               const uint32_t* __restrict__ hist, int nblk) {
+  __shared__ uint32_t base[256];
+  __shared__ uint32_t wcnt[kSortThreads / 32][256];
+  int64_t lo;
+  const int64_t n = resolve_n(ns, &lo);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  base[threadIdx.x] = hist[(size_t)threadIdx.x * nblk + blockIdx.x];
+#pragma unroll
+  for (int w = 0; w < kSortThreads / 32; ++w) wcnt[w][threadIdx.x] = 0;
+  __syncthreads();
+  const int64_t tile0 = (int64_t)blockIdx.x * kSortTile;
+  if (tile0 >= n) return;
+  for (int r = 0; r < kSortRounds; ++r) {
+    const int64_t i = tile0 + r * kSortThreads + threadIdx.x;
+    const bool valid = i < n;
+    uint64_t k = 0;
+    uint32_t src = 0;
+    if (valid) {
+      k = keys_in[i];
+      src = idx_in ? idx_in[i] : (uint32_t)i;
+    }
+    const uint32_t d = (uint32_t)(k >> shift) & 255u;
+    const uint32_t tag = valid ? d : (256u + (uint32_t)lane);  // invalid lanes match nobody
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, tag);
+    const uint32_t rank = __popc(peers & ((1u << lane) - 1u));
+    if (valid && rank == 0) wcnt[warp][d] = __popc(peers);
+    __syncthreads();
+    if (valid) {
+      uint32_t pos = base[d] + rank;
+      for (int w = 0; w < warp; ++w) pos += wcnt[w][d];
+      keys_out[pos] = k;
+      idx_out[pos] = src;
+    }
+    __syncthreads();
+    uint32_t add = 0;
+#pragma unroll
+    for (int w = 0; w < kSortThreads / 32; ++w) {
+      add += wcnt[w][threadIdx.x];
+      wcnt[w][threadIdx.x] = 0;
+    }
+    base[threadIdx.x] += add;
+    __syncthreads();
+  }
+}
+
+// ---- unique / inverse / probe ---------------------------------------------
+
+__device__ __forceinline__ int32_t cache_probe(const CacheDev& c, int64_t key) {
+  if (c.n == 0) return -1;
+  const uint32_t b = (uint32_t)((uint64_t)key >> c.bucket_shift);
+  uint32_t lo = c.bucket_start[b], hi = c.bucket_start[b + 1];
+  while (lo < hi) {
+    const uint32_t mid = (lo + hi) >> 1;
+    const int64_t v = c.keys[mid];
+    if (v == key) return (int32_t)mid;
+    if (v < key) lo = mid + 1;
+    else hi = mid;
+  }
+  return -1;
+}
+
+// Block-wide exclusive scan of one value per thread (256 threads); returns the
+// exclusive prefix and the block total.
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* total, uint32_t* sh /*[8]*/) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+    if (lane >= d) inc += t;
+  }
+  __syncthreads();  // sh may still be in use by a previous call
+  if (lane == 31) sh[warp] = inc;
+  __syncthreads();
+  uint32_t before = 0, all = 0;
+#pragma unroll
+  for (int w = 0; w < kScanThreads / 32; ++w) {
+    const uint32_t s = sh[w];
+    if (w < warp) before += s;
+    all += s;
+  }
+  *total = all;
+  return before + inc - v;
+}
+
+// Pass 1: count heads (first of each run of equal keys) per tile; with PROBE
+// also look every head up in the cache, remember the answer per sorted
+// position and count the misses.
+template <bool PROBE>
+__global__ void __launch_bounds__(kScanThreads) unique_count_kernel(NSrc ns, const uint64_t* __restrict__ keys,
+                                                                    CacheDev cache, int32_t* __restrict__ probe_tmp,
+                                                                    uint32_t* __restrict__ tile_counts, int nblk) {
+  __shared__ uint32_t sh[8];
+  int64_t lo;
+  const int64_t n = resolve_n(ns, &lo);
+  const int64_t i0 = ((int64_t)blockIdx.x * kScanThreads + threadIdx.x) * kScanItems;
+  uint32_t heads = 0, misses = 0;
+#pragma unroll
+  for (int j = 0; j < kScanItems; ++j) {
+    const int64_t i = i0 + j;
+    if (i < n) {
+      const uint64_t k = keys[i];
+      const bool head = (i == 0) || (keys[i - 1] != k);
+      if (head) {
+        ++heads;
+        if (PROBE) {
+          const int32_t slot = cache_probe(cache, (int64_t)k);
+          probe_tmp[i] = slot;
+          if (slot < 0) ++misses;
+        }
+      }
+    }
+  }
+  uint32_t th, tm;
+  block_excl_scan(heads, &th, sh);
+  if (PROBE) block_excl_scan(misses, &tm, sh);
+  if (threadIdx.x == 0) {
+    tile_counts[blockIdx.x] = th;
+    if (PROBE) tile_counts[nblk + blockIdx.x] = tm;
+  }
+}
+
+// Pass 2 (one block): exclusive scan of the per-tile counts; totals out.
+__global__ void __launch_bounds__(1024) unique_scan_kernel(uint32_t* __restrict__ tile_counts, int nblk, int n_arrays,
+                                                           int64_t* __restrict__ n_unique, int64_t* __restrict__ n_miss) {
+  __shared__ uint32_t warp_sum[32];
+  for (int a = 0; a < n_arrays; ++a) {
+    uint32_t* arr = tile_counts + (size_t)a * nblk;
+    const int per = (nblk + 1023) / 1024;
+    const int begin = min(nblk, (int)threadIdx.x * per), end = min(nblk, begin + per);
+    uint32_t sum = 0;
+    for (int i = begin; i < end; ++i) sum += arr[i];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+      if (lane >= d) inc += t;
+    }
+    __syncthreads();
+    if (lane == 31) warp_sum[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t w = warp_sum[lane];
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, w, d);
+        if (lane >= d) w += t;
+      }
+      warp_sum[lane] = w;
+    }
+    __syncthreads();
+    uint32_t run = inc - sum + (warp ? warp_sum[warp - 1] : 0u);
+    for (int i = begin; i < end; ++i) {
+      const uint32_t v = arr[i];
+      arr[i] = run;
+      run += v;
+    }
+    if (threadIdx.x == 1023) {
+      if (a == 0) *n_unique = (int64_t)run;
+      else *n_miss = (int64_t)run;
+    }
+  }
+}
+
+// Pass 3: write uniq, inverse and (PROBE) the per-unique source and the list of
+// missed rows.
+template <bool PROBE>
+__global__ void __launch_bounds__(kScanThreads) unique_write_kernel(NSrc ns, const uint64_t* __restrict__ keys,
+                                                                    const uint32_t* __restrict__ idx,
+                                                                    const int32_t* __restrict__ probe_tmp,
+                                                                    const uint32_t* __restrict__ tile_counts, int nblk,
+                                                                    int64_t* __restrict__ uniq, int32_t* __restrict__ inverse,
+                                                                    int32_t* __restrict__ src, int64_t* __restrict__ miss_rows) {
+  __shared__ uint32_t sh[8];
+  int64_t lo;
+  const int64_t n = resolve_n(ns, &lo);
+  const int64_t i0 = ((int64_t)blockIdx.x * kScanThreads + threadIdx.x) * kScanItems;
+  uint64_t k[kScanItems];
+  bool head[kScanItems];
+  int32_t slot[kScanItems];
+  uint32_t heads = 0, misses = 0;
+#pragma unroll
+  for (int j = 0; j < kScanItems; ++j) {
+    const int64_t i = i0 + j;
+    head[j] = false;
+    slot[j] = 0;
+    k[j] = 0;
+    if (i < n) {
+      k[j] = keys[i];
+      head[j] = (i == 0) || (keys[i - 1] != k[j]);
+      if (head[j]) {
+        ++heads;
+        if (PROBE) {
+          slot[j] = probe_tmp[i];
+          if (slot[j] < 0) ++misses;
+        }
+      }
+    }
+  }
+  uint32_t tot;
+  uint32_t u = tile_counts[blockIdx.x] + block_excl_scan(heads, &tot, sh);
+  uint32_t m = 0;
+  if (PROBE) m = tile_counts[nblk + blockIdx.x] + block_excl_scan(misses, &tot, sh);
+  // u = number of heads strictly before this thread's first element
+#pragma unroll
+  for (int j = 0; j < kScanItems; ++j) {
+    const int64_t i = i0 + j;
+    if (i < n) {
+      if (head[j]) {
+        uniq[u] = (int64_t)k[j];
+        if (PROBE) {
+          if (slot[j] < 0) {
+            src[u] = -1 - (int32_t)m;
+            miss_rows[m] = (int64_t)k[j];
+            ++m;
+          } else {
+            src[u] = slot[j];
+          }
+        }
+        ++u;
+      }
+      inverse[idx[i]] = (int32_t)(u - 1);
+    }
+  }
+}
+
+inline uint64_t align256(uint64_t x) { return (x + 255u) & ~255ULL; }
+
+}  // namespace
+
+uint64_t workspace_layout(int64_t max_ids, uint64_t max_row_bytes, WsLayout* L) {
+  WsLayout l;
+  const uint64_t n = (uint64_t)(max_ids > 0 ? max_ids : 0);
+  l.nblk_sort = (int)((n + kSortTile - 1) / kSortTile);
+  l.nblk_scan = (int)((n + kScanTile - 1) / kScanTile);
+  if (l.nblk_sort < 1) l.nblk_sort = 1;
+  if (l.nblk_scan < 1) l.nblk_scan = 1;
+  uint64_t off = 0;
+  auto take = [&](uint64_t bytes) {
+    const uint64_t at = off;
+    off = align256(off + bytes);
+    return at;
+  };
+  l.keys_a = take(n * 8);
+  l.keys_b = take(n * 8);
+  l.idx_a = take(n * 4);
+  l.idx_b = take(n * 4);
+  l.hist = take((uint64_t)l.nblk_sort * 256 * 4);
+  l.tile_counts = take((uint64_t)l.nblk_scan * 2 * 4);
+  l.counters = take(64);
+  l.uniq = take(n * 8);
+  l.inverse = take(n * 4);
+  l.src = take(n * 4);
+  l.miss_rows = take(n * 8);
+  l.staging = take(n * max_row_bytes);
+  l.total = off;
+  if (L) *L = l;
+  return off;
+}
+
+// Sort + unique + inverse (+ cache probe). `first_keys` is the array that pass 0
+// reads when hash == nullptr; with hash != nullptr pass 0 hashes the slot's raw
+// IDs into the workspace instead. On return (in stream order) uniq / inverse /
+// n_unique hold the dedup result; with `cache` non-null also src / miss_rows /
+// n_miss.
+cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s) {
+  uint8_t* ws = (uint8_t*)a.ws;
+  const WsLayout& L = a.layout;
+  uint64_t* ka = (uint64_t*)(ws + L.keys_a);
+  uint64_t* kb = (uint64_t*)(ws + L.keys_b);
+  uint32_t* ia = (uint32_t*)(ws + L.idx_a);
+  uint32_t* ib = (uint32_t*)(ws + L.idx_b);
+  uint32_t* hist = (uint32_t*)(ws + L.hist);
+  uint32_t* tile_counts = (uint32_t*)(ws + L.tile_counts);
+
+  const int64_t cap = a.ns.offsets ? a.ns.cap : a.ns.n_imm;
+  const int nblk = (int)((cap + kSortTile - 1) / kSortTile) > 0 ? (int)((cap + kSortTile - 1) / kSortTile) : 1;
+  const int nblk2 = (int)((cap + kScanTile - 1) / kScanTile) > 0 ? (int)((cap + kScanTile - 1) / kScanTile) : 1;
+  int bits = 1;
+  while (bits < 63 && (a.max_key >> bits) != 0) ++bits;
+  const int passes = (bits + 7) / 8;
+
+  const uint64_t* kin = a.hash ? ka : a.first_keys;
+  const uint32_t* iin = nullptr;
+  uint64_t* kout = a.hash ? kb : ka;
+  uint32_t* iout = ia;
+  for (int p = 0; p < passes; ++p) {
+    const int shift = 8 * p;
+    if (p == 0 && a.hash)
+      hist_kernel<true><<<nblk, kSortThreads, 0, s>>>(a.ns, nullptr, ka, a.hash->ids, a.hash->seed, a.hash->rows,
+                                                      a.hash->magic, a.hash->pre_hashed, shift, hist, nblk, a.err);
+    else
+      hist_kernel<false><<<nblk, kSortThreads, 0, s>>>(a.ns, kin, nullptr, nullptr, 0, 0, 0, 0, shift, hist, nblk, a.err);
+    scan_counters_kernel<<<1, 1024, 0, s>>>(hist, 256 * nblk);
+    scatter_kernel<<<nblk, kSortThreads, 0, s>>>(a.ns, kin, iin, kout, iout, shift, hist, nblk);
+    *launches += 3;
+    // next pass reads what this one wrote
+    kin = kout;
+    iin = iout;
+    kout = (kout == ka) ? kb : ka;
+    iout = (iout == ia) ? ib : ia;
+  }
+  // kin / iin: sorted keys and their original positions; iout is free
+  int32_t* probe_tmp = (int32_t*)iout;
+  if (a.cache) {
+    unique_count_kernel<true><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, *a.cache, probe_tmp, tile_counts, nblk2);
+    unique_scan_kernel<<<1, 1024, 0, s>>>(tile_counts, nblk2, 2, a.n_unique, a.n_miss);
+    unique_write_kernel<true><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, iin, probe_tmp, tile_counts, nblk2, a.uniq,
+                                                            a.inverse, a.src, a.miss_rows);
+  } else {
+    CacheDev none{};
+    unique_count_kernel<false><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, none, nullptr, tile_counts, nblk2);
+    unique_scan_kernel<<<1, 1024, 0, s>>>(tile_counts, nblk2, 1, a.n_unique, nullptr);
+    unique_write_kernel<false><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, iin, nullptr, tile_counts, nblk2, a.uniq,
+                                                             a.inverse, nullptr, nullptr);
+  }
+  *launches += 3;
+  return cudaGetLastError();
+}
+
+}  // namespace mfet

@@ -1,0 +1,515 @@
+"""GPU parity: every result of the CUDA library is compared with the CPU oracle on
+the same seeded inputs, through the C-ABI binding. Indices and dedup output are
+bit-exact; pooled fp32 outputs are within |gpu - ref| <= 1e-6 + 1e-5*|ref|."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2508_05700_b200 import inputs as gi
+from tests.helpers import (DeviceTables, assert_close, forward, mfet, workload_forward, workload_oracle)
+
+pytestmark = pytest.mark.gpu
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+# ------------------------------------------------------------------ hash ----
+
+@pytest.mark.parametrize("rows", [1, 7, 100_000, 10_000_000, 50_000_000, 10**9, 2**32 - 1, 2**32, 2**32 + 1,
+                                  2**40 + 12345, 2**63 - 1])
+def test_hash_ids_bit_exact(rows):
+    m = mfet()
+    rng = np.random.default_rng(rows % 1000)
+    n = 300_001
+    ids = rng.integers(0, 2**64 - 1, size=n, dtype=np.uint64)
+    ids[:6] = [0, 1, 2, 2**40 - 1, 2**63, 2**64 - 1]
+    seed = 0 if rows in (1, 100_000) else 0x5DEECE66D1234567
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    h = m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), rows, 4, m.F32, m.LOC_DEVICE, 0, seed, 0)])
+    try:
+        d_ids = torch.from_numpy(ids.view(np.int64)).cuda()
+        d_rows = torch.empty(n, dtype=torch.int64, device="cuda")
+        m.mfet_hash_ids(h, 0, d_ids, n, d_rows, _stream())
+        got = d_rows.cpu().numpy()
+        assert np.array_equal(got, orc.hash_ids(ids, seed, rows))
+        # in place
+        m.mfet_hash_ids(h, 0, d_ids, n, d_ids, _stream())
+        assert np.array_equal(d_ids.cpu().numpy(), got)
+        m.mfet_hash_ids(h, 0, None, 0, None, _stream())  # n = 0 is a no-op
+    finally:
+        m.mfet_tables_destroy(h)
+
+
+# ------------------------------------------------------------------ fill ----
+
+@pytest.mark.parametrize("dtype", [gi.F32, gi.F16, gi.BF16])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_table_fill_bit_exact(dtype, mode):
+    m = mfet()
+    rows, dim, key = 5003, 40, 0x1234ABCD9876FEDB
+    rb = m.row_bytes(dim, dtype)
+    buf = torch.zeros(rows * rb, dtype=torch.uint8, device="cuda")
+    m.mfet_table_fill(buf, 0, rows, dim, dtype, 0, key, mode, _stream())
+    got = buf.cpu().numpy().reshape(rows, rb)
+    want = orc.table_fill(orc.Table(rows=rows, dim=dim, dtype=dtype, value_key=key, value_mode=mode))
+    assert np.array_equal(got, want)
+    # a sub-range (rows 4000..4099 land at data + r*stride) with a padded stride
+    stride = rb + 32
+    buf2 = torch.zeros(100 * stride, dtype=torch.uint8, device="cuda")
+    m.mfet_table_fill(buf2.data_ptr() - 4000 * stride, 4000, 100, dim, dtype, stride, key, mode, _stream())
+    got2 = buf2.cpu().numpy().reshape(100, stride)
+    assert np.array_equal(got2[:, :rb], want[4000:4100])
+    assert not got2[:, rb:].any()
+
+
+def test_table_fill_frozen_literals():
+    m = mfet()
+    with open(os.path.join(GOLD, "table_values.txt")) as fh:
+        for line in fh:
+            if line.startswith("#") or not line.strip():
+                continue
+            key, mode, dim, dtype, r, d, bits = (int(x, 0) for x in line.split())
+            rb = m.row_bytes(dim, dtype)
+            buf = torch.zeros(rb, dtype=torch.uint8, device="cuda")
+            m.mfet_table_fill(buf.data_ptr() - r * rb, r, 1, dim, dtype, 0, key, mode, _stream())
+            raw = buf.cpu().numpy()
+            got = int(raw.view(np.uint32)[d]) if dtype == gi.F32 else int(raw.view(np.uint16)[d])
+            assert got == bits, line
+
+
+# ----------------------------------------------------------- dtype decode ---
+
+@pytest.mark.parametrize("dtype", [gi.F16, gi.BF16])
+def test_decode_all_16bit_patterns(dtype):
+    """Every finite 16-bit pattern decodes on the GPU to the oracle's fp32 bits
+    (single-ID bags, pre-hashed row indices, so the output is the row itself)."""
+    m = mfet()
+    pat = np.arange(65536, dtype=np.uint16).reshape(8192, 8)
+    tab = torch.from_numpy(pat.view(np.int16).copy()).cuda()
+    h = m.mfet_tables_create([m.TableDesc(tab.data_ptr(), 8192, 8, dtype, m.LOC_DEVICE, 0, 0, 0)])
+    try:
+        ids = torch.arange(8192, dtype=torch.int64, device="cuda")
+        off = torch.arange(8193, dtype=torch.int64, device="cuda")
+        out = torch.empty(8192, 8, dtype=torch.float32, device="cuda")
+        shape, keep = m.make_shape(8192, 1, [0], ids_are_rows=True)
+        m.mfet_embedding_bag_forward(h, shape, ids, off, None, [0], [m.POOL_SUM], out, _stream())
+        got = out.cpu().numpy().view(np.uint32).reshape(-1)
+    finally:
+        m.mfet_tables_destroy(h)
+    conv = orc.f16_bits_to_f32_bits if dtype == gi.F16 else orc.bf16_bits_to_f32_bits
+    want = np.array([conv(int(x)) for x in range(65536)], np.uint32)
+    finite = np.isfinite(want.view(np.float32)) & (want != 0x80000000)  # 0 + (-0) = +0 on both sides
+    assert np.array_equal(got[finite], want[finite])
+    assert (got[want == 0x80000000] == 0).all()
+
+
+# ------------------------------------------------------------ tiny cases ----
+
+def _mat_tables(tabs, dtypes, seeds=None):
+    """Materialised tables (numpy fp32 [rows, dim]) -> (device handle pieces, oracle tables)."""
+    m = mfet()
+    dev, descs, otabs = [], [], []
+    for i, (x, dt) in enumerate(zip(tabs, dtypes)):
+        x = np.ascontiguousarray(x, np.float32)
+        if dt == gi.F32:
+            raw = x
+        elif dt == gi.F16:
+            raw = x.astype(np.float16)
+        else:
+            raw = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy()
+        raw = np.ascontiguousarray(raw)
+        d = torch.from_numpy(raw.view(np.uint8).reshape(-1).copy()).cuda()
+        seed = seeds[i] if seeds else 0
+        dev.append(d)
+        descs.append(m.TableDesc(d.data_ptr(), x.shape[0], x.shape[1], dt, m.LOC_DEVICE, 0, seed, 0))
+        otabs.append(orc.Table(rows=x.shape[0], dim=x.shape[1], dtype=dt, hash_seed=seed, data=raw))
+    return dev, descs, otabs
+
+
+class _Mat:
+    def __init__(self, tabs, dtypes, seeds=None):
+        self.m = mfet()
+        self.dev, descs, self.oracle_tables = _mat_tables(tabs, dtypes, seeds)
+        self.specs = [gi.TableSpec(t.shape[0], t.shape[1], dt, 0, 0) for t, dt in zip(tabs, dtypes)]
+        self.h = self.m.mfet_tables_create(descs)
+
+    def close(self):
+        torch.cuda.synchronize()
+        self.m.mfet_tables_destroy(self.h)
+
+
+@pytest.mark.parametrize("dtype", [gi.F32, gi.F16, gi.BF16])
+def test_hand_computed_tiny_bags(dtype):
+    g = {}
+    with open(os.path.join(GOLD, "tiny_bags.txt")) as fh:
+        for line in fh:
+            if not line.startswith("#") and line.strip():
+                k, *v = line.split()
+                g[k] = np.array([float(x) for x in v])
+    D = 8  # rows must be a multiple of 16 bytes: the 2 real columns are padded with zeros
+    tab = np.zeros((4, D), np.float32)
+    tab[:, :2] = g["table"].reshape(4, 2)
+    mt = _Mat([tab], [dtype])
+    try:
+        for pool, key in ((0, "sum"), (1, "mean"), (2, "wsum")):
+            out = forward(mt, 3, 1, [0], [0], [pool], g["ids"].astype(np.uint64), g["offsets"].astype(np.int64),
+                          g["weights"].astype(np.float32), ids_are_rows=True)
+            assert np.array_equal(out[:, :2], g[key].reshape(3, 2).astype(np.float32)), key
+            assert not out[:, 2:].any()
+    finally:
+        mt.close()
+
+
+def _ragged(rng, n_bags, pattern):
+    if pattern == "mixed":
+        lens = rng.integers(0, 12, size=n_bags)
+        lens[rng.random(n_bags) < 0.25] = 0
+        lens[rng.integers(0, n_bags, 5)] = rng.integers(33, 300, 5)
+    elif pattern == "ones":
+        lens = np.ones(n_bags, np.int64)
+    elif pattern == "empty_edges":
+        lens = rng.integers(1, 9, size=n_bags)
+        lens[0] = lens[-1] = lens[n_bags // 2] = 0
+    elif pattern == "all_empty":
+        lens = np.zeros(n_bags, np.int64)
+    elif pattern == "long":
+        lens = rng.integers(30, 700, size=n_bags)
+    else:
+        raise ValueError(pattern)
+    off = np.zeros(n_bags + 1, np.int64)
+    np.cumsum(lens, out=off[1:])
+    return off
+
+
+@pytest.mark.parametrize("dtype,dim", [(gi.F32, 4), (gi.F32, 32), (gi.F32, 20), (gi.F16, 8), (gi.F16, 64),
+                                       (gi.BF16, 32), (gi.BF16, 64), (gi.BF16, 128), (gi.BF16, 24),
+                                       (gi.F16, 256), (gi.F32, 128), (gi.BF16, 520), (gi.F32, 260)])
+@pytest.mark.parametrize("pattern", ["mixed", "ones", "empty_edges", "all_empty", "long"])
+@pytest.mark.parametrize("policy", [0, 1, 2])
+def test_unit_parity(dtype, dim, pattern, policy):
+    rng = np.random.default_rng(dim * 7 + dtype)
+    rows = 16 if pattern != "long" else 977
+    B = 77 if pattern != "long" else 19
+    tab = (0.01 * rng.standard_normal((rows, dim))).astype(np.float32)  # the workloads' value scale
+    mt = _Mat([tab], [dtype], seeds=[0xABCDEF])
+    try:
+        mt.m.mfet_set_option(mt.h, mt.m.OPT_GROUP_POLICY, policy)
+        off = _ragged(rng, B, pattern)
+        ids = rng.integers(0, 2**40, size=int(off[-1]), dtype=np.uint64)
+        if ids.size > 4:
+            ids[1] = ids[0]  # duplicate inside a bag
+        w = rng.random(ids.size).astype(np.float32)
+        for pool in (0, 1, 2):
+            got = forward(mt, B, 1, [0], [0], [pool], ids, off, w)
+            ref = orc.embedding_bag(mt.oracle_tables, B, 1, [0], [0], [pool], ids, off, w)
+            assert_close(got, ref, "pool %d" % pool)
+            lens = np.diff(off)
+            assert not got[lens == 0].any()
+    finally:
+        mt.close()
+
+
+def test_single_row_table_and_prehashed_rows():
+    rng = np.random.default_rng(3)
+    tab = rng.standard_normal((1, 32)).astype(np.float32)
+    mt = _Mat([tab], [gi.F32], seeds=[77])
+    try:
+        off = np.array([0, 3, 3, 10], np.int64)
+        ids = rng.integers(0, 2**40, size=10, dtype=np.uint64)
+        got = forward(mt, 3, 1, [0], [0], [0], ids, off, None)
+        assert_close(got, np.stack([3 * tab[0], 0 * tab[0], 7 * tab[0]]))
+    finally:
+        mt.close()
+
+
+def test_grid_tables_are_bit_exact_in_any_order():
+    """Grid-valued tables make every unweighted sum exact in fp32, so GPU and oracle agree bit for bit."""
+    w = gi.make_workload(2, rows_scale=1e-3, batch_scale=1 / 16)
+    with DeviceTables(w.tables, value_mode=1) as dt:
+        b = gi.make_batch(w, 0)
+        sums = np.array([gi.POOL_SUM] * w.n_slots, np.int32)
+        for policy in (0, 1, 2):
+            dt.m.mfet_set_option(dt.h, dt.m.OPT_GROUP_POLICY, policy)
+            got = forward(dt, w.batch, w.n_features, w.slot_feature, w.table_ids, sums, b.ids, b.offsets, None)
+            ref = orc.embedding_bag(dt.oracle_tables, w.batch, w.n_features, w.slot_feature, w.table_ids, sums,
+                                    b.ids, b.offsets, None)
+            assert np.array_equal(got, ref)
+
+
+# --------------------------------------------------------------- workloads --
+
+SCALED = {1: (1.0, 1.0), 2: (0.01, 0.25), 3: (0.004, 0.125), 4: (0.005, 1 / 32), 5: (0.002, 0.125)}
+
+
+@pytest.mark.parametrize("config", [1, 2, 3, 4])
+def test_workload_parity_scaled(config):
+    rs, bs = SCALED[config]
+    w = gi.make_workload(config, rows_scale=rs, batch_scale=bs)
+    with DeviceTables(w.tables) as dt:
+        for j in (0, 1):
+            b = gi.make_batch(w, j)
+            got = workload_forward(dt, w, b)
+            ref = workload_oracle(dt, w, b)
+            assert_close(got, ref, "config %d batch %d" % (config, j))
+        # bit-identical on a second run (fixed summation order)
+        again = workload_forward(dt, w, b)
+        assert np.array_equal(got, again)
+
+
+def test_facets_concat_equals_single_slot_calls():
+    w = gi.make_workload(3, rows_scale=0.002, batch_scale=1 / 16)
+    with DeviceTables(w.tables) as dt:
+        b = gi.make_batch(w, 0)
+        full = workload_forward(dt, w, b)
+        col = 0
+        for s in range(w.n_slots):
+            D = w.tables[int(w.table_ids[s])].dim
+            one = forward(dt, w.batch, w.n_features, [int(w.slot_feature[s])], [int(w.table_ids[s])],
+                          [int(w.pooling[s])], b.ids, b.offsets, b.weights)
+            assert np.array_equal(full[:, col:col + D], one)
+            col += D
+        assert col == 896
+
+
+def test_output_leading_dimension_and_unaligned_out():
+    w = gi.make_workload(3, rows_scale=0.001, batch_scale=1 / 64)
+    with DeviceTables(w.tables) as dt:
+        b = gi.make_batch(w, 0)
+        ref = workload_oracle(dt, w, b)
+        wide = workload_forward(dt, w, b, out_ld=900)
+        assert_close(wide[:, :896], ref)
+        assert np.isnan(wide[:, 896:]).all()  # columns beyond the slots are left alone
+        odd = workload_forward(dt, w, b, out_ld=899)  # rows not 16-byte aligned: scalar stores
+        assert_close(odd[:, :896], ref)
+        # an output base that is only 4-byte aligned
+        big = torch.full((w.batch * 896 + 1,), float("nan"), dtype=torch.float32, device="cuda")
+        view = big[1:].view(w.batch, 896)
+        got = workload_forward(dt, w, b, out=view)
+        assert_close(got, ref)
+
+
+def test_many_slots_need_several_launches():
+    rng = np.random.default_rng(5)
+    tabs = [(0.01 * rng.standard_normal((50, 8))).astype(np.float32) for _ in range(4)]
+    mt = _Mat(tabs, [gi.F32, gi.F16, gi.BF16, gi.F32], seeds=[1, 2, 3, 4])
+    try:
+        B, F, L = 33, 3, 130
+        off = _ragged(rng, F * B, "mixed")
+        ids = rng.integers(0, 2**40, size=int(off[-1]), dtype=np.uint64)
+        w = rng.random(ids.size).astype(np.float32)
+        sf = np.sort(rng.integers(0, F, L)).astype(np.int32)
+        ti = rng.integers(0, 4, L).astype(np.int32)
+        po = rng.integers(0, 3, L).astype(np.int32)
+        got = forward(mt, B, F, sf, ti, po, ids, off, w)
+        ref = orc.embedding_bag(mt.oracle_tables, B, F, sf, ti, po, ids, off, w)
+        assert_close(got, ref)
+    finally:
+        mt.close()
+
+
+def test_forward_host_equals_forward():
+    m = mfet()
+    w = gi.make_workload(2, rows_scale=0.001, batch_scale=1 / 16)
+    with DeviceTables(w.tables) as dt:
+        b = gi.make_batch(w, 0)
+        ref = workload_forward(dt, w, b)
+        shape, keep = m.make_shape(w.batch, w.n_features, w.slot_feature)
+        nnz = int(b.offsets[-1])
+        nbytes = m.mfet_host_io_bytes(dt.h, shape, w.table_ids, nnz)
+        io = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        ids_h = torch.from_numpy(b.ids.view(np.int64)).pin_memory()
+        off_h = torch.from_numpy(b.offsets).pin_memory()
+        out_h = torch.empty(w.batch, w.out_dim, dtype=torch.float32).pin_memory()
+        m.mfet_embedding_bag_forward_host(dt.h, shape, ids_h, off_h, None, nnz, w.table_ids, w.pooling, out_h, io,
+                                          nbytes, _stream())
+        assert np.array_equal(out_h.numpy(), ref)
+
+
+# ------------------------------------------------------------------ dedup ---
+
+@pytest.mark.parametrize("n,hi", [(0, 10), (1, 10), (2, 2), (255, 10**9), (256, 10**9), (257, 50), (2047, 10**9),
+                                  (2048, 3), (2049, 10**6), (4096, 1), (65537, 10**9), (300_000, 10**9),
+                                  (300_000, 2**62), (100_000, 70_000)])
+def test_dedup_bit_exact(n, hi):
+    m = mfet()
+    rng = np.random.default_rng(n + hi % 97)
+    rows = rng.integers(0, hi, size=n, dtype=np.int64)
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    h = m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), 8, 4, m.F32, m.LOC_DEVICE, 0, 0, 0)])
+    try:
+        cap = max(n, 1) + 100
+        ws = torch.empty(m.mfet_workspace_bytes(h, cap), dtype=torch.uint8, device="cuda")
+        m.mfet_set_workspace(h, ws, ws.numel(), cap)
+        d_rows = torch.from_numpy(rows).cuda()
+        uniq = torch.full((max(n, 1),), -7, dtype=torch.int64, device="cuda")
+        inv = torch.full((max(n, 1),), -7, dtype=torch.int32, device="cuda")
+        nu = torch.full((1,), -7, dtype=torch.int64, device="cuda")
+        for max_row in (0, hi):
+            m.mfet_dedup_rows(h, d_rows, n, uniq, inv, nu, max_row, _stream())
+            torch.cuda.synchronize()
+            wu, wi = orc.dedup(rows)
+            k = int(nu.item())
+            assert k == wu.size
+            assert np.array_equal(uniq.cpu().numpy()[:k], wu)
+            assert np.array_equal(inv.cpu().numpy()[:n], wi)
+            assert np.array_equal(d_rows.cpu().numpy(), rows)  # input untouched
+        assert m.mfet_query_status(h) == 0
+    finally:
+        m.mfet_tables_destroy(h)
+
+
+# -------------------------------------------------------------- host path ---
+
+def _hot_rows(dt, w, table_id, feature, count, rows_total):
+    """Hashed rows of the `count` hottest IDs of a feature (hashing done by the library), first
+    distinct rows in popularity order, returned sorted."""
+    m = dt.m
+    ids = gi.hot_ids(w, feature, count)
+    d = torch.from_numpy(ids.view(np.int64)).cuda()
+    r = torch.empty_like(d)
+    m.mfet_hash_ids(dt.h, table_id, d, d.numel(), r, _stream())
+    rows = r.cpu().numpy()
+    _, first = np.unique(rows, return_index=True)
+    keep = rows[np.sort(first)]
+    return np.sort(keep)
+
+
+@pytest.mark.parametrize("pinned_by_caller", [True, False])
+def test_host_table_path_matches_oracle_and_hbm_placement(pinned_by_caller):
+    w = gi.make_workload(5, rows_scale=0.002, batch_scale=0.125)  # host table: 2M rows x 64 fp16 = 256 MB
+    b = gi.make_batch(w, 0)
+    n_host = int(b.offsets[w.batch] - b.offsets[0])
+    with DeviceTables(w.tables, host_pinned=pinned_by_caller) as dt:
+        dt.set_workspace(int(n_host * 1.25) + 1024)
+        ref = workload_oracle(dt, w, b)
+        cold = workload_forward(dt, w, b)           # no cache: every distinct row crosses PCIe
+        assert_close(cold, ref, "host path, no cache")
+        hot = _hot_rows(dt, w, 0, 0, int(w.tables[0].rows * w.cache_fraction), w.tables[0].rows)
+        dt.build_cache(0, hot)
+        warm = workload_forward(dt, w, b)           # cache on
+        assert np.array_equal(warm, cold)
+        b1 = gi.make_batch(w, 1)
+        assert_close(workload_forward(dt, w, b1), workload_oracle(dt, w, b1), "host path, cache on")
+        dt.build_cache(0, np.arange(0, w.tables[0].rows, dtype=np.int64))  # everything cached
+        assert np.array_equal(workload_forward(dt, w, b), cold)
+        launches = dt.m.mfet_launch_count(dt.h)
+        assert launches > 0
+    # the same table placed in HBM gives the same bits
+    specs = [gi.TableSpec(t.rows, t.dim, t.dtype, t.hash_seed, t.value_key, gi.LOC_DEVICE) for t in w.tables]
+    with DeviceTables(specs) as dt2:
+        hbm = workload_forward(dt2, w, b)
+    assert_close(hbm, ref)
+    assert np.array_equal(hbm[:, 64:], cold[:, 64:])
+    assert_close(hbm[:, :64], cold[:, :64])
+
+
+def test_host_slot_over_workspace_capacity_sets_error_bit():
+    w = gi.make_workload(5, rows_scale=0.0005, batch_scale=1 / 64)
+    b = gi.make_batch(w, 0)
+    with DeviceTables(w.tables) as dt:
+        dt.set_workspace(16)  # far too small for the host feature
+        m = dt.m
+        out = torch.full((w.batch, w.out_dim), float("nan"), dtype=torch.float32, device="cuda")
+        shape, keep = m.make_shape(w.batch, w.n_features, w.slot_feature)
+        m.mfet_embedding_bag_forward(dt.h, shape, torch.from_numpy(b.ids.view(np.int64)).cuda(),
+                                     torch.from_numpy(b.offsets).cuda(), None, w.table_ids, w.pooling, out, _stream())
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(dt.h, clear=True) & m.DEV_CAPACITY
+        assert m.mfet_query_status(dt.h) == 0
+        got = out.cpu().numpy()
+        assert not got[:, :64].any()  # the over-capacity slot is written as zeros
+        assert_close(got[:, 64:], workload_oracle(dt, w, b)[:, 64:])
+
+
+# ----------------------------------------------------------- host-side errors
+
+def test_argument_errors_are_reported_before_any_launch():
+    m = mfet()
+    dummy = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    good = m.TableDesc(dummy.data_ptr(), 8, 4, m.F32, m.LOC_DEVICE, 0, 0, 0)
+
+    def status(fn, *a, **k):
+        try:
+            fn(*a, **k)
+        except m.MfetError as e:
+            return e.status
+        return 0
+
+    assert status(m.mfet_tables_create, [m.TableDesc(dummy.data_ptr(), 0, 4, m.F32, 0, 0, 0, 0)]) == m.ERR_INVALID_ARG
+    assert status(m.mfet_tables_create, [m.TableDesc(None, 8, 4, m.F32, 0, 0, 0, 0)]) == m.ERR_INVALID_ARG
+    assert status(m.mfet_tables_create, [m.TableDesc(dummy.data_ptr(), 8, 3, m.F32, 0, 0, 0, 0)]) == m.ERR_UNSUPPORTED_DIM
+    assert status(m.mfet_tables_create, [m.TableDesc(dummy.data_ptr() + 4, 8, 4, m.F32, 0, 0, 0, 0)]) == m.ERR_ALIGNMENT
+    assert status(m.mfet_tables_create, [m.TableDesc(dummy.data_ptr(), 8, 4, m.F32, 0, 0, 0, 24)]) == m.ERR_ALIGNMENT
+    assert status(m.mfet_tables_create, [m.TableDesc(dummy.data_ptr(), 8, 4, 9, 0, 0, 0, 0)]) == m.ERR_INVALID_ARG
+    assert status(m.mfet_tables_create, [good], 9999) == m.ERR_INVALID_ARG
+    host = m.TableDesc(None, 64, 8, m.F16, m.LOC_HOST, 0, 0, 0)
+    h = m.mfet_tables_create([good, host])
+    try:
+        launches = m.mfet_launch_count(h)
+        ids = torch.zeros(4, dtype=torch.int64, device="cuda")
+        off = torch.tensor([0, 2, 4], dtype=torch.int64, device="cuda")
+        out = torch.zeros(2, 4, device="cuda")
+        sh, k = m.make_shape(2, 1, [0])
+        assert status(m.mfet_embedding_bag_forward, h, sh, ids, off, None, [5], [0], out) == m.ERR_INVALID_ARG
+        assert status(m.mfet_embedding_bag_forward, h, sh, ids, off, None, [0], [3], out) == m.ERR_INVALID_ARG
+        assert status(m.mfet_embedding_bag_forward, h, sh, ids, off, None, [0], [m.POOL_WSUM], out) == m.ERR_INVALID_ARG
+        assert status(m.mfet_embedding_bag_forward, h, sh, None, off, None, [0], [0], out) == m.ERR_INVALID_ARG
+        assert status(m.mfet_embedding_bag_forward, h, sh, ids, off, None, [1], [0], out) == m.ERR_NOT_REGISTERED
+        sh2, k2 = m.make_shape(2, 1, [0], out_ld=2)
+        assert status(m.mfet_embedding_bag_forward, h, sh2, ids, off, None, [0], [0], out) == m.ERR_INVALID_ARG
+        sh3, k3 = m.make_shape(2, 1, [1])
+        assert status(m.mfet_embedding_bag_forward, h, sh3, ids, off, None, [0], [0], out) == m.ERR_INVALID_ARG
+        assert status(m.mfet_hash_ids, h, 7, ids, 4, ids) == m.ERR_INVALID_ARG
+        assert status(m.mfet_host_tables_register, h, 0, dummy.data_ptr(), 4096) == m.ERR_INVALID_ARG
+        pinned = torch.zeros(64 * 16, dtype=torch.uint8).pin_memory()
+        assert status(m.mfet_host_tables_register, h, 1, pinned.data_ptr(), 100, 1) == m.ERR_INVALID_ARG
+        assert status(m.mfet_host_tables_register, h, 1, pinned.data_ptr() + 8, 1016, 1) == m.ERR_ALIGNMENT
+        assert status(m.mfet_cache_build, h, 1, np.array([1, 2], np.int64), dummy, 4096) == m.ERR_NOT_REGISTERED
+        m.mfet_host_tables_register(h, 1, pinned.data_ptr(), pinned.numel(), 1)
+        assert status(m.mfet_host_tables_register, h, 1, pinned.data_ptr(), pinned.numel(), 1) == m.ERR_INVALID_ARG
+        assert status(m.mfet_embedding_bag_forward, h, sh, ids, off, None, [1], [0],
+                      torch.zeros(2, 8, device="cuda")) == m.ERR_WORKSPACE
+        assert status(m.mfet_cache_build, h, 1, np.array([2, 1], np.int64), dummy, 4096) == m.ERR_INVALID_ARG
+        assert status(m.mfet_cache_build, h, 1, np.array([1, 64], np.int64), dummy, 4096) == m.ERR_INVALID_ARG
+        assert status(m.mfet_cache_build, h, 1, np.array([1, 2], np.int64), dummy, 16) == m.ERR_WORKSPACE
+        assert status(m.mfet_set_workspace, h, dummy.data_ptr() + 16, 4000, 4) == m.ERR_ALIGNMENT
+        assert status(m.mfet_set_workspace, h, dummy, 256, 1000) == m.ERR_WORKSPACE
+        assert status(m.mfet_dedup_rows, h, ids, 4, ids, ids, ids, 0) == m.ERR_WORKSPACE
+        assert status(m.mfet_set_option, h, 99, 0) == m.ERR_INVALID_ARG
+        assert m.mfet_launch_count(h) == launches  # nothing was launched by any rejected call
+        assert m.mfet_query_status(h) == 0
+    finally:
+        m.mfet_tables_destroy(h)
+    assert "workspace" in m.status_string(m.ERR_WORKSPACE)
+
+
+def test_device_error_bits_for_bad_prehashed_rows_and_offsets():
+    rng = np.random.default_rng(1)
+    tab = rng.standard_normal((16, 8)).astype(np.float32)
+    mt = _Mat([tab], [gi.F32])
+    try:
+        m = mt.m
+        ids = torch.tensor([1, 99, 2], dtype=torch.int64, device="cuda")  # 99 >= rows
+        off = torch.tensor([0, 3], dtype=torch.int64, device="cuda")
+        out = torch.empty(1, 8, device="cuda")
+        sh, k = m.make_shape(1, 1, [0], ids_are_rows=True)
+        m.mfet_embedding_bag_forward(mt.h, sh, ids, off, None, [0], [0], out)
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(mt.h, clear=True) == m.DEV_ROW_RANGE
+        assert_close(out.cpu().numpy()[0], tab[1] + tab[2])  # the bad index is skipped
+        off_bad = torch.tensor([0, 3, 1], dtype=torch.int64, device="cuda")
+        out2 = torch.empty(2, 8, device="cuda")
+        sh2, k2 = m.make_shape(2, 1, [0], ids_are_rows=True)
+        ids2 = torch.tensor([1, 3, 2], dtype=torch.int64, device="cuda")
+        m.mfet_embedding_bag_forward(mt.h, sh2, ids2, off_bad, None, [0], [0], out2)
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(mt.h, clear=True) == m.DEV_OFFSETS
+        assert not out2.cpu().numpy()[1].any()
+    finally:
+        mt.close()
