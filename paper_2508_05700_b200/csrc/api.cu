@@ -61,8 +61,7 @@ int mfet_tables_create(const mfet_table_desc_t* descs, int32_t n_tables, int32_t
   for (int32_t i = 0; i < n_tables; ++i) {
     const mfet_table_desc_t& d = descs[i];
     if (d.rows == 0 || d.rows >= (1ULL << 63) || d.dim == 0 || d.flags != 0) return MFET_ERR_INVALID_ARG;
-    if (d.dtype > MFET_INT4 || d.location > MFET_LOC_HOST) return MFET_ERR_INVALID_ARG;
-    if (d.dtype == MFET_INT4 && (d.dim & 1u)) return MFET_ERR_UNSUPPORTED_DIM;
+    if (d.dtype > MFET_BF16 || d.location > MFET_LOC_HOST) return MFET_ERR_INVALID_ARG;
     const uint64_t rb = mfet_row_bytes(d.dim, d.dtype);
     if (rb == 0 || rb % 16 != 0) return MFET_ERR_UNSUPPORTED_DIM;
     const uint64_t stride = d.row_stride_bytes ? d.row_stride_bytes : rb;
@@ -170,9 +169,9 @@ int mfet_hash_ids(const mfet_tables_t* t, int32_t table_id, const uint64_t* ids,
 int mfet_table_fill(void* data, uint64_t row0, uint64_t n_rows, uint32_t dim, uint32_t dtype,
                     uint64_t row_stride_bytes, uint64_t value_key, uint32_t value_mode,
                     mfet_stream_t stream) {
-  if (!data || dim == 0 || dtype > MFET_INT4 || value_mode > MFET_VAL_GRID) return MFET_ERR_INVALID_ARG;
+  if (!data || dim == 0 || dtype > MFET_BF16 || value_mode > MFET_VAL_GRID) return MFET_ERR_INVALID_ARG;
   const uint64_t rb = mfet_row_bytes(dim, dtype);
-  if (rb == 0 || rb % 16 != 0 || (dtype == MFET_INT4 && (dim & 1u))) return MFET_ERR_UNSUPPORTED_DIM;
+  if (rb == 0 || rb % 16 != 0) return MFET_ERR_UNSUPPORTED_DIM;
   const uint64_t stride = row_stride_bytes ? row_stride_bytes : rb;
   if (stride < rb) return MFET_ERR_INVALID_ARG;
   if (stride % 16 != 0 || !aligned16(data)) return MFET_ERR_ALIGNMENT;
