@@ -167,6 +167,33 @@ MFET_API int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape
 MFET_API int mfet_dedup_rows(mfet_tables_t* t, const int64_t* rows, int64_t n, int64_t* uniq,
                     int32_t* inverse, int64_t* n_unique, int64_t max_row, mfet_stream_t stream);
 
+/* The same dedup for callers that have no device memory to lend and must not
+ * ask the driver for any. (This entry point has no counterpart in the paper; it
+ * exists for embedding the library in hosts with a closed memory budget.)
+ * Typical cases: a plug-in running inside a serving process whose whole GPU
+ * memory was handed to another allocator at start-up, so a later cudaMalloc
+ * fails or evicts somebody else's pool; a latency-critical request thread, for
+ * which cudaMalloc/cudaFree are off limits because they synchronise the whole
+ * device; code that holds no table handle and therefore no workspace.
+ * Nothing is allocated here, by the library or on its behalf: the sort's
+ * scratch is a fixed array compiled into the library, about 6.1 MiB that every
+ * GPU using the library holds until the process ends. Hence the limit:
+ *   0 <= n <= MFET_STATIC_DEDUP_MAX_IDS, otherwise MFET_ERR_WORKSPACE (use
+ *   mfet_dedup_rows with a workspace for larger batches).
+ * device: CUDA ordinal of the GPU that owns rows/uniq/inverse/n_unique (0..63);
+ * the other arguments and the result are those of mfet_dedup_rows, bit for bit.
+ * The first call on each GPU looks up the device address of the built-in array
+ * (a runtime query, once per GPU); make that first call outside any stream
+ * capture. All calls on a GPU share the one array and it keeps whatever the
+ * previous call left (each call overwrites what it reads, nothing needs
+ * clearing): two calls whose kernels can overlap on the GPU - different
+ * streams without an ordering, or several host threads - race on it and give
+ * wrong results; order them on one stream or with events.
+ * Errors: INVALID_ARG, WORKSPACE (n too large), CUDA. */
+#define MFET_STATIC_DEDUP_MAX_IDS 262144
+MFET_API int mfet_dedup_rows_static(int32_t device, const int64_t* rows, int64_t n, int64_t* uniq,
+                           int32_t* inverse, int64_t* n_unique, int64_t max_row, mfet_stream_t stream);
+
 /* Device bytes that the hot-row cache of `n` rows of table `table_id` needs. */
 MFET_API int mfet_cache_bytes(const mfet_tables_t* t, int32_t table_id, int64_t n, uint64_t* bytes /*host*/);
 

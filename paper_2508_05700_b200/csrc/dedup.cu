@@ -6,6 +6,9 @@
 // Every kernel here is a plain data-parallel pass; the passes are ordered by the
 // stream, so no kernel ever waits on another block. Results are canonical
 // (ascending unique rows), hence bit-reproducible.
+#include <cstring>
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mfet {
@@ -442,3 +445,93 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
 }
 
 }  // namespace mfet
+
+// ---- dedup without any caller- or library-side allocation -------------------
+//
+// The sort's ping-pong buffers and counters live in a fixed device array that
+// is part of the library image: every GPU that loads the library holds these
+// bytes until the process exits, which is why the capacity is kept modest.
+
+namespace {
+
+constexpr int64_t kStaticMaxIds = MFET_STATIC_DEDUP_MAX_IDS;
+constexpr uint64_t kStaticSortBlocks = (kStaticMaxIds + mfet::kSortTile - 1) / mfet::kSortTile;
+constexpr uint64_t kStaticScanBlocks = (kStaticMaxIds + mfet::kScanTile - 1) / mfet::kScanTile;
+constexpr uint64_t pad256(uint64_t x) { return (x + 255u) & ~255ULL; }
+constexpr uint64_t kOffKeysA = 0;
+constexpr uint64_t kOffKeysB = kOffKeysA + pad256(kStaticMaxIds * 8);
+constexpr uint64_t kOffIdxA = kOffKeysB + pad256(kStaticMaxIds * 8);
+constexpr uint64_t kOffIdxB = kOffIdxA + pad256(kStaticMaxIds * 4);
+constexpr uint64_t kOffHist = kOffIdxB + pad256(kStaticMaxIds * 4);
+constexpr uint64_t kOffTiles = kOffHist + pad256(kStaticSortBlocks * 256 * 4);
+constexpr uint64_t kStaticScratchBytes = kOffTiles + pad256(kStaticScanBlocks * 2 * 4);
+
+// In host code this name is only a handle of the symbol, not a device address:
+// the address is asked from the runtime once per device (below).
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices];  // device address of g_static_scratch, per GPU
+bool g_scratch_ready[kMaxDevices];
+std::mutex g_scratch_mutex;
+
+}  // namespace
+
+extern "C" int mfet_dedup_rows_static(int32_t device, const int64_t* rows, int64_t n, int64_t* uniq,
+                                      int32_t* inverse, int64_t* n_unique, int64_t max_row,
+                                      mfet_stream_t stream_) {
+  if (device < 0 || device >= kMaxDevices || n < 0 || !n_unique || max_row < 0) return MFET_ERR_INVALID_ARG;
+  if (n > kStaticMaxIds) return MFET_ERR_WORKSPACE;  // beyond the built-in scratch: use mfet_dedup_rows
+  if (n > 0 && (!rows || !uniq || !inverse)) return MFET_ERR_INVALID_ARG;
+  int prev = 0;
+  if (cudaGetDevice(&prev) != cudaSuccess) return MFET_ERR_CUDA;
+  if (prev != device && cudaSetDevice(device) != cudaSuccess) {
+    cudaGetLastError();
+    return MFET_ERR_INVALID_ARG;
+  }
+  cudaStream_t stream = (cudaStream_t)stream_;
+  int rc = MFET_OK;
+  void* scratch = nullptr;
+  {
+    // first call on this GPU: look the array's device address up, with this GPU current
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ready[device]) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+        cudaGetLastError();
+        rc = MFET_ERR_CUDA;
+      } else {
+        g_scratch_addr[device] = p;
+        g_scratch_ready[device] = true;
+      }
+    }
+    scratch = g_scratch_addr[device];
+  }
+  if (rc == MFET_OK) {
+    if (n == 0) {
+      if (cudaMemsetAsync(n_unique, 0, sizeof(int64_t), stream) != cudaSuccess) rc = MFET_ERR_CUDA;
+    } else {
+      // every scratch region that a pass reads is written in full by an earlier pass of the
+      // same call, so nothing left over from the previous call needs clearing
+      mfet::DedupArgs a;
+      std::memset(&a, 0, sizeof(a));
+      a.ns = mfet::NSrc{nullptr, 0, 0, n, n};
+      a.first_keys = reinterpret_cast<const uint64_t*>(rows);
+      a.max_key = max_row > 0 ? (uint64_t)max_row - 1 : 0x7FFFFFFFFFFFFFFFULL;
+      a.ws = scratch;
+      a.layout.keys_a = kOffKeysA;
+      a.layout.keys_b = kOffKeysB;
+      a.layout.idx_a = kOffIdxA;
+      a.layout.idx_b = kOffIdxB;
+      a.layout.hist = kOffHist;
+      a.layout.tile_counts = kOffTiles;
+      a.uniq = uniq;
+      a.inverse = inverse;
+      a.n_unique = n_unique;
+      uint64_t launches = 0;
+      if (mfet::launch_dedup(a, &launches, stream) != cudaSuccess) rc = MFET_ERR_CUDA;
+    }
+  }
+  if (prev != device) cudaSetDevice(prev);
+  return rc;
+}

@@ -32,8 +32,9 @@ EXPORTS = [
     "mfet_hash_ids", "mfet_embedding_bag_forward", "mfet_dedup_rows", "mfet_cache_bytes",
     "mfet_cache_build", "mfet_workspace_bytes", "mfet_set_workspace", "mfet_host_io_bytes",
     "mfet_embedding_bag_forward_host", "mfet_table_fill", "mfet_query_status", "mfet_set_option",
-    "mfet_launch_count", "mfet_status_string",
+    "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static",
 ]
+STATIC_DEDUP_MAX_IDS = 262144
 
 
 class TableDesc(C.Structure):
@@ -63,6 +64,7 @@ _lib.mfet_host_tables_register.argtypes = [_P, C.c_int32, _P, C.c_uint64, C.c_ui
 _lib.mfet_hash_ids.argtypes = [_P, C.c_int32, _P, C.c_int64, _P, _P]
 _lib.mfet_embedding_bag_forward.argtypes = [_P, C.POINTER(BatchShape), _P, _P, _P, _P, _P, _P, _P]
 _lib.mfet_dedup_rows.argtypes = [_P, _P, C.c_int64, _P, _P, _P, C.c_int64, _P]
+_lib.mfet_dedup_rows_static.argtypes = [C.c_int32, _P, C.c_int64, _P, _P, _P, C.c_int64, _P]
 _lib.mfet_cache_bytes.argtypes = [_P, C.c_int32, C.c_int64, C.POINTER(C.c_uint64)]
 _lib.mfet_cache_build.argtypes = [_P, C.c_int32, _P, C.c_int64, _P, C.c_uint64, _P]
 _lib.mfet_workspace_bytes.argtypes = [_P, C.c_int64, C.POINTER(C.c_uint64)]
@@ -154,6 +156,13 @@ def mfet_embedding_bag_forward(h, shape: BatchShape, ids, offsets, weights, tabl
 def mfet_dedup_rows(h, rows, n: int, uniq, inverse, n_unique, max_row: int = 0, stream=None) -> None:
     _check(_lib.mfet_dedup_rows(h, _ptr(rows), n, _ptr(uniq), _ptr(inverse), _ptr(n_unique), max_row,
                                 _ptr(stream)), "mfet_dedup_rows")
+
+
+def mfet_dedup_rows_static(device: int, rows, n: int, uniq, inverse, n_unique, max_row: int = 0, stream=None) -> None:
+    """Dedup on the library's built-in scratch array: no workspace, no allocation anywhere
+    (n <= STATIC_DEDUP_MAX_IDS). Calls on one GPU share that array and must not overlap."""
+    _check(_lib.mfet_dedup_rows_static(device, _ptr(rows), n, _ptr(uniq), _ptr(inverse), _ptr(n_unique), max_row,
+                                       _ptr(stream)), "mfet_dedup_rows_static")
 
 
 def mfet_cache_bytes(h, table_id: int, n: int) -> int:
