@@ -47,7 +47,7 @@ enum { MFET_F32 = 0, MFET_F16 = 1, MFET_BF16 = 2, MFET_INT4 = 3 };
 enum { MFET_POOL_SUM = 0, MFET_POOL_MEAN = 1, MFET_POOL_WSUM = 2 };
 enum { MFET_LOC_DEVICE = 0, MFET_LOC_HOST = 1 };
 enum { MFET_VAL_NORMAL = 0, MFET_VAL_GRID = 1 };
-enum { MFET_OPT_GROUP_POLICY = 1 };
+enum { MFET_OPT_GROUP_POLICY = 1, MFET_OPT_TILE = 2 };
 
 enum {
   MFET_OK = 0,
@@ -250,7 +250,9 @@ MFET_API int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits /*h
 /* Tuning knobs. MFET_OPT_GROUP_POLICY: how the pooling kernel maps lanes to
  * bags: 0 = chosen per tile from its mean bag length (default), 1 = one row
  * group per bag (best for short bags), 2 = one warp per bag (long bags). The
- * result is the same up to the order of fp32 additions. */
+ * result is the same up to the order of fp32 additions. MFET_OPT_TILE: samples per
+ * thread block of the pooling kernel: 0 = chosen from the batch size (default), or
+ * 8 / 16 / 32 / 64. */
 MFET_API int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value);
 
 /* Number of kernels the library has launched on behalf of this handle. */

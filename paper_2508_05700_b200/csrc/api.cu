@@ -200,6 +200,10 @@ int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value) {
       if (value < 0 || value > 2) return MFET_ERR_INVALID_ARG;
       t->group_policy = (int32_t)value;
       return MFET_OK;
+    case MFET_OPT_TILE:
+      if (value != 0 && value != 8 && value != 16 && value != 32 && value != 64) return MFET_ERR_INVALID_ARG;
+      t->tile = (int32_t)value;
+      return MFET_OK;
     default: return MFET_ERR_INVALID_ARG;
   }
 }
@@ -281,6 +285,7 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
   // bags per block: full tiles once there is enough work to fill the GPU several times over
   const int64_t bags = (int64_t)B * L;
   p.tile = bags >= 148LL * 8 * 64 ? 64 : (bags >= 148LL * 4 * 32 ? 32 : 16);
+  if (t->tile) p.tile = t->tile;
   p.tiles_per_slot = (B + p.tile - 1) / p.tile;
 
   // host-table slots go to the side stream, forked from and joined to `stream`

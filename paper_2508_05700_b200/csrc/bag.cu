@@ -18,11 +18,24 @@
 // the tile configuration, never on timing.
 #include "common.cuh"
 
+// Tunables (overridable at build time for sweeps): row loads kept in flight per
+// lane, and the minimum number of resident blocks per SM that caps registers.
+#ifndef MFET_BAG_U
+#define MFET_BAG_U 4
+#endif
+#ifndef MFET_BAG_LONG
+#define MFET_BAG_LONG 64
+#endif
+#ifndef MFET_BAG_MINB
+#define MFET_BAG_MINB 4
+#endif
+
 namespace mfet {
 
 namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
+constexpr int kLongBag = MFET_BAG_LONG;  // bags at least this long get a whole warp
 
 template <int DT>
 struct ChunkElems {
@@ -89,11 +102,12 @@ struct ReduceScatter {
 //              slot's feature, so that positions are slot-local).
 template <int DT, int LPR, int GL, bool IND>
 __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, const int64_t* soff,
-                                          int b0, int nb, const IndirectParams& ip, int64_t feat_lo) {
+                                          int b0, const uint8_t* perm, int q0, int q1,
+                                          const IndirectParams& ip, int64_t feat_lo) {
   constexpr int E = ChunkElems<DT>::value;
   constexpr int GG = GL / LPR;          // row groups per bag group
   constexpr int NG = 256 / GL;          // bag groups per block
-  constexpr int U = LPR < 4 ? LPR : 4;  // row loads in flight per lane
+  constexpr int U = LPR < MFET_BAG_U ? LPR : MFET_BAG_U;  // row loads in flight per lane
   constexpr int NF = (E / GG) > 0 ? (E / GG) : 1;  // values a lane stores
 
   const int lane = threadIdx.x & 31;
@@ -109,11 +123,15 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
   const uint64_t stride16 = s.stride >> 4;
   const unsigned long long* ids = reinterpret_cast<const unsigned long long*>(p.ids);
 
-  for (int it = 0; it * NG < p.tile; ++it) {
-    const int bi = it * NG + grp;
+  // bags perm[q0 .. q1) of the tile, NG at a time (perm orders the tile by falling length,
+  // so the bag groups of one warp work on bags of similar length)
+  for (int qb = q0; qb < q1; qb += NG) {
+    const int q = qb + grp;
+    const bool have = q < q1;
+    const int bi = have ? (int)perm[q] : 0;
     int64_t lo = 0;
     int len = 0;
-    if (bi < nb) {
+    if (have) {
       lo = soff[bi];
       int64_t l = soff[bi + 1] - lo;
       if (l < 0) {
@@ -178,7 +196,7 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
     }
 
     int off = 0;
-    bool writer = (bi < nb) && chunk_ok;
+    bool writer = have && chunk_ok;
     ReduceScatter<E, 0, GG, LPR>::run(acc, sub, off, writer);
     if (s.pooling == MFET_POOL_MEAN && len > 0) {
       const float fl = (float)len;
@@ -205,30 +223,31 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
   }
 }
 
-#define MFET_POOL_ARGS p, s, soff, b0, nb, ip, feat_lo
+#define MFET_POOL_ARGS p, s, soff, b0, perm, ip, feat_lo
 
+// Bags perm[0 .. n_long) are long: one warp each. The rest: one row group each.
 template <int DT, int LPR, bool IND>
 __device__ __forceinline__ void pool_tile_lpr(const BagParams& p, const SlotDev& s, const int64_t* soff,
-                                              int b0, int nb, const IndirectParams& ip, int64_t feat_lo,
-                                              bool warp_mode) {
+                                              int b0, const uint8_t* perm, const IndirectParams& ip,
+                                              int64_t feat_lo, int n_long, int nb) {
   if constexpr (LPR == 32) {
-    pool_tile<DT, 32, 32, IND>(MFET_POOL_ARGS);
+    pool_tile<DT, 32, 32, IND>(p, s, soff, b0, perm, 0, nb, ip, feat_lo);
   } else {
-    if (warp_mode) pool_tile<DT, LPR, 32, IND>(MFET_POOL_ARGS);
-    else pool_tile<DT, LPR, LPR, IND>(MFET_POOL_ARGS);
+    if (n_long > 0) pool_tile<DT, LPR, 32, IND>(p, s, soff, b0, perm, 0, n_long, ip, feat_lo);
+    if (n_long < nb) pool_tile<DT, LPR, LPR, IND>(p, s, soff, b0, perm, n_long, nb, ip, feat_lo);
   }
 }
 
 template <int DT, bool IND>
 __device__ __forceinline__ void pool_tile_dt(const BagParams& p, const SlotDev& s, const int64_t* soff,
-                                             int b0, int nb, const IndirectParams& ip, int64_t feat_lo,
-                                             bool warp_mode) {
+                                             int b0, const uint8_t* perm, const IndirectParams& ip,
+                                             int64_t feat_lo, int n_long, int nb) {
   switch (s.lpr_log2) {
-    case 1: pool_tile_lpr<DT, 2, IND>(MFET_POOL_ARGS, warp_mode); break;
-    case 2: pool_tile_lpr<DT, 4, IND>(MFET_POOL_ARGS, warp_mode); break;
-    case 3: pool_tile_lpr<DT, 8, IND>(MFET_POOL_ARGS, warp_mode); break;
-    case 4: pool_tile_lpr<DT, 16, IND>(MFET_POOL_ARGS, warp_mode); break;
-    default: pool_tile_lpr<DT, 32, IND>(MFET_POOL_ARGS, warp_mode); break;
+    case 1: pool_tile_lpr<DT, 2, IND>(MFET_POOL_ARGS, n_long, nb); break;
+    case 2: pool_tile_lpr<DT, 4, IND>(MFET_POOL_ARGS, n_long, nb); break;
+    case 3: pool_tile_lpr<DT, 8, IND>(MFET_POOL_ARGS, n_long, nb); break;
+    case 4: pool_tile_lpr<DT, 16, IND>(MFET_POOL_ARGS, n_long, nb); break;
+    default: pool_tile_lpr<DT, 32, IND>(MFET_POOL_ARGS, n_long, nb); break;
   }
 }
 
@@ -236,6 +255,8 @@ template <bool IND>
 __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParams& ip) {
   __shared__ int64_t soff[kMaxTile + 1];
   __shared__ int64_t sfeat[2];
+  __shared__ uint8_t perm[kMaxTile];
+  __shared__ int scnt[2][16];
   const int slot = blockIdx.x / p.tiles_per_slot;
   const int tile = blockIdx.x - slot * p.tiles_per_slot;
   const SlotDev& s = p.slot[slot];
@@ -244,6 +265,7 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   const long long* offs = reinterpret_cast<const long long*>(p.offsets) + (int64_t)s.feature * p.batch;
   if ((int)threadIdx.x <= nb) soff[threadIdx.x] = __ldcs(offs + b0 + threadIdx.x);
   if (IND && threadIdx.x < 2) sfeat[threadIdx.x] = offs[threadIdx.x ? p.batch : 0];
+  if (threadIdx.x >= 128 && threadIdx.x < 160) (&scnt[0][0])[threadIdx.x - 128] = 0;
   __syncthreads();
   int64_t feat_lo = 0;
   if constexpr (IND) {
@@ -258,25 +280,47 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
     }
   }
 
-  // one warp per bag once the tile's mean bag fills a warp's round reasonably
-  const int64_t total = soff[nb] - soff[0];
-  bool warp_mode = total >= (int64_t)nb * 24;
-  if (p.group_policy == 1) warp_mode = false;
-  if (p.group_policy == 2) warp_mode = true;
+  // Order the tile's bags by falling length class (counting sort over 16 classes, stable
+  // inside a class): class 15 = long bags (a whole warp each), classes 0..14 = shorter ones
+  // in steps of kLongBag/15, so that the bag groups of one warp get bags of similar length.
+  const int lane_ = threadIdx.x & 31, warp_ = threadIdx.x >> 5;
+  bool have = false;
+  int cls = 0, in_warp = 0;
+  if (warp_ < 2) {  // threads 0..63 own one bag each
+    have = (int)threadIdx.x < nb;
+    if (have) {
+      const int64_t l = soff[threadIdx.x + 1] - soff[threadIdx.x];
+      const int len = l < 0 ? 0 : (l > 0x7FFFFFFF ? 0x7FFFFFFF : (int)l);
+      cls = len >= kLongBag ? 15 : (len * 15) / kLongBag;
+    }
+    const unsigned peers = __match_any_sync(kFull, have ? cls : 16 + lane_);
+    in_warp = __popc(peers & ((1u << lane_) - 1u));
+    if (have && in_warp == 0) scnt[warp_][cls] = __popc(peers);
+  }
+  __syncthreads();
+  if (have) {
+    int rank = in_warp + (warp_ ? scnt[0][cls] : 0);
+    for (int c2 = cls + 1; c2 < 16; ++c2) rank += scnt[0][c2] + scnt[1][c2];
+    perm[rank] = (uint8_t)threadIdx.x;
+  }
+  __syncthreads();
+  int n_long = scnt[0][15] + scnt[1][15];
+  if (p.group_policy == 1) n_long = 0;
+  if (p.group_policy == 2) n_long = nb;
 
   switch (s.dtype) {
-    case MFET_F32: pool_tile_dt<MFET_F32, IND>(MFET_POOL_ARGS, warp_mode); break;
-    case MFET_F16: pool_tile_dt<MFET_F16, IND>(MFET_POOL_ARGS, warp_mode); break;
-    default: pool_tile_dt<MFET_BF16, IND>(MFET_POOL_ARGS, warp_mode); break;
+    case MFET_F32: pool_tile_dt<MFET_F32, IND>(MFET_POOL_ARGS, n_long, nb); break;
+    case MFET_F16: pool_tile_dt<MFET_F16, IND>(MFET_POOL_ARGS, n_long, nb); break;
+    default: pool_tile_dt<MFET_BF16, IND>(MFET_POOL_ARGS, n_long, nb); break;
   }
 }
 
-__global__ void __launch_bounds__(256) bag_kernel(const __grid_constant__ BagParams p) {
+__global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_kernel(const __grid_constant__ BagParams p) {
   const IndirectParams none{};
   bag_body<false>(p, none);
 }
 
-__global__ void __launch_bounds__(256) bag_indirect_kernel(const __grid_constant__ BagParams p,
+__global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_indirect_kernel(const __grid_constant__ BagParams p,
                                                            const __grid_constant__ IndirectParams ip) {
   bag_body<true>(p, ip);
 }

@@ -51,6 +51,7 @@ struct mfet_tables {
   int64_t ws_max_ids = 0;
   uint64_t launches = 0;
   int32_t group_policy = 0;
+  int32_t tile = 0;  // bags per block; 0 = chosen from the batch size
 };
 
 namespace mfet {
