@@ -47,7 +47,7 @@ enum { MFET_F32 = 0, MFET_F16 = 1, MFET_BF16 = 2, MFET_INT4 = 3 };
 enum { MFET_POOL_SUM = 0, MFET_POOL_MEAN = 1, MFET_POOL_WSUM = 2 };
 enum { MFET_LOC_DEVICE = 0, MFET_LOC_HOST = 1 };
 enum { MFET_VAL_NORMAL = 0, MFET_VAL_GRID = 1 };
-enum { MFET_OPT_GROUP_POLICY = 1, MFET_OPT_TILE = 2 };
+enum { MFET_OPT_GROUP_POLICY = 1, MFET_OPT_TILE = 2, MFET_OPT_PROFILE = 3 };
 
 enum {
   MFET_OK = 0,
@@ -252,8 +252,15 @@ MFET_API int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits /*h
  * group per bag (best for short bags), 2 = one warp per bag (long bags). The
  * result is the same up to the order of fp32 additions. MFET_OPT_TILE: samples per
  * thread block of the pooling kernel: 0 = chosen from the batch size (default), or
- * 8 / 16 / 32 / 64. */
+ * 8 / 16 / 32 / 64. MFET_OPT_PROFILE: 1 = record CUDA events around the stages of
+ * the host-table path of every forward call (read them with mfet_profile_read). */
 MFET_API int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value);
+
+/* Stage times of the host-table path of the most recent forward call that had a
+ * host-table slot, in milliseconds: stage_ms[0] hash + dedup + cache probe,
+ * [1] fetch of the missed rows from host memory, [2] pooling. Waits for that
+ * call's host-table path to finish. Needs MFET_OPT_PROFILE = 1 (else INVALID_ARG). */
+MFET_API int mfet_profile_read(mfet_tables_t* t, float* stage_ms /*host float[3]*/);
 
 /* Number of kernels the library has launched on behalf of this handle. */
 MFET_API int mfet_launch_count(const mfet_tables_t* t, uint64_t* launches /*host*/);

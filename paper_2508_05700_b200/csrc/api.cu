@@ -114,6 +114,8 @@ int mfet_tables_destroy(mfet_tables_t* t) {
   }
   if (t->ev_fork) cudaEventDestroy(t->ev_fork);
   if (t->ev_join) cudaEventDestroy(t->ev_join);
+  for (int i = 0; i < 4; ++i)
+    if (t->prof_ev[i]) cudaEventDestroy(t->prof_ev[i]);
   for (TableHost& tb : t->tables)
     if (tb.pinned_by_us && tb.host_ptr) cudaHostUnregister(tb.host_ptr);
   if (t->err_host) cudaFreeHost(t->err_host);
@@ -200,12 +202,32 @@ int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value) {
       if (value < 0 || value > 2) return MFET_ERR_INVALID_ARG;
       t->group_policy = (int32_t)value;
       return MFET_OK;
+    case MFET_OPT_PROFILE:
+      if (value != 0 && value != 1) return MFET_ERR_INVALID_ARG;
+      if (value == 1 && !t->prof_ev[0]) {
+        DeviceGuard g(t->device);
+        for (int i = 0; i < 4; ++i)
+          if (cudaEventCreate(&t->prof_ev[i]) != cudaSuccess) return MFET_ERR_CUDA;
+      }
+      t->profile = (int32_t)value;
+      t->prof_valid = false;
+      return MFET_OK;
     case MFET_OPT_TILE:
       if (value != 0 && value != 8 && value != 16 && value != 32 && value != 64) return MFET_ERR_INVALID_ARG;
       t->tile = (int32_t)value;
       return MFET_OK;
     default: return MFET_ERR_INVALID_ARG;
   }
+}
+
+int mfet_profile_read(mfet_tables_t* t, float* stage_ms) {
+  if (!t || !stage_ms) return MFET_ERR_INVALID_ARG;
+  if (!t->profile || !t->prof_valid) return MFET_ERR_INVALID_ARG;
+  DeviceGuard g(t->device);
+  if (cudaEventSynchronize(t->prof_ev[3]) != cudaSuccess) return MFET_ERR_CUDA;
+  for (int i = 0; i < 3; ++i)
+    if (cudaEventElapsedTime(&stage_ms[i], t->prof_ev[i], t->prof_ev[i + 1]) != cudaSuccess) return MFET_ERR_CUDA;
+  return MFET_OK;
 }
 
 int mfet_workspace_bytes(const mfet_tables_t* t, int64_t max_ids, uint64_t* bytes) {

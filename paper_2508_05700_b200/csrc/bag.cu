@@ -2,24 +2,31 @@
 // slots of a batch in one launch.
 //
 // Work split. A block takes one (slot, tile of up to 64 consecutive samples);
-// the tile's CSR offsets are staged in shared memory. Inside the block a BAG
-// GROUP of GL lanes owns one bag at a time. A row of the table is 16-byte
-// chunks; LPR lanes (a ROW GROUP) read one row with one 16-byte load each, so a
-// bag group reads GL/LPR rows per load instruction. GL is either LPR (short
-// bags: no cross-lane reduction at all, several bags per warp) or 32 (long
-// bags: the whole warp streams one bag), chosen per tile from its mean length.
+// the tile's CSR offsets are staged in shared memory and its bags are ordered by
+// falling length class. Inside the block a BAG GROUP of GL lanes owns one bag at
+// a time. A table row is 16-byte chunks; LPR lanes (a ROW GROUP) read one row
+// with one 16-byte load each, so a bag group reads GL/LPR rows per load
+// instruction. Long bags get GL = 32 (the whole warp streams one bag), all other
+// bags GL = LPR (several bags per warp, no cross-lane reduction at all); thanks
+// to the ordering the bag groups of a warp work on bags of similar length.
 //
-// Per round a bag group takes GL IDs: every lane loads and hashes one ID
-// (coalesced 8-byte loads, all lanes busy), then the row offsets travel by
-// shuffle to the row group that loads them, U loads in flight per lane.
-// Accumulation is fp32; row groups are combined by a shuffle reduce-scatter so
-// that every lane ends with a distinct piece of the output row and the store is
-// one coalesced segment. The order of additions depends only on the inputs and
-// the tile configuration, never on timing.
+// The work of a bag group is a sequence of ROUNDS of GL IDs. In a round every
+// lane hashes one ID (coalesced 8-byte loads, prefetched one round ahead so the
+// ID latency hides behind the previous round's rows), the row offsets travel by
+// shuffle to the row group that loads them, U loads are in flight per lane, and
+// batches of loads whose rows exist in every bag group of the warp run without
+// predicates. Accumulation is fp32 (packed two-wide FMA); row groups are
+// combined by a shuffle reduce-scatter so that every lane ends with a distinct
+// piece of the output row and the store is one coalesced segment. The order of
+// additions depends only on the inputs and the tile configuration, never on
+// timing.
 #include "common.cuh"
 
 // Tunables (overridable at build time for sweeps): row loads kept in flight per
-// lane, and the minimum number of resident blocks per SM that caps registers.
+// lane, the length from which a bag gets a whole warp, the minimum number of
+// resident blocks per SM (caps registers) and the accumulate flavour
+// (0 convert + scalar FMA, 1 packed f32x2 FMA, 2 mixed-precision add for
+// unweighted 16-bit tables).
 #ifndef MFET_BAG_U
 #define MFET_BAG_U 4
 #endif
@@ -27,7 +34,10 @@
 #define MFET_BAG_LONG 64
 #endif
 #ifndef MFET_BAG_MINB
-#define MFET_BAG_MINB 4
+#define MFET_BAG_MINB 5
+#endif
+#ifndef MFET_BAG_ACC
+#define MFET_BAG_ACC 1
 #endif
 
 namespace mfet {
@@ -42,30 +52,73 @@ struct ChunkElems {
   static constexpr int value = (DT == MFET_F32) ? 4 : 8;
 };
 
-// acc += w * (the 16-byte chunk v decoded to fp32); exact up-conversion.
+__device__ __forceinline__ unsigned long long pack2(uint32_t lo, uint32_t hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+
+// a += x * w on two packed fp32 lanes (each lane one IEEE fused multiply-add).
+__device__ __forceinline__ void fma2(unsigned long long& a, unsigned long long x, unsigned long long w) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(a) : "l"(x), "l"(w));
+}
+
+// acc (E fp32 values as E/2 packed pairs) += w * (the 16-byte chunk v decoded to
+// fp32). The up-conversion of fp16 / bf16 is exact.
 template <int DT>
-__device__ __forceinline__ void accumulate(float* acc, const uint4& v, float w) {
+__device__ __forceinline__ void accumulate(unsigned long long* acc, const uint4& v, float w, bool wsum) {
+  const uint32_t x[4] = {v.x, v.y, v.z, v.w};
+#if MFET_BAG_ACC == 0
+  float* a = reinterpret_cast<float*>(acc);
   if constexpr (DT == MFET_F32) {
-    acc[0] = fmaf(w, __uint_as_float(v.x), acc[0]);
-    acc[1] = fmaf(w, __uint_as_float(v.y), acc[1]);
-    acc[2] = fmaf(w, __uint_as_float(v.z), acc[2]);
-    acc[3] = fmaf(w, __uint_as_float(v.w), acc[3]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) a[j] = fmaf(w, __uint_as_float(x[j]), a[j]);
   } else if constexpr (DT == MFET_F16) {
-    const uint32_t x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&x[j]));
-      acc[2 * j] = fmaf(w, f.x, acc[2 * j]);
-      acc[2 * j + 1] = fmaf(w, f.y, acc[2 * j + 1]);
+      a[2 * j] = fmaf(w, f.x, a[2 * j]);
+      a[2 * j + 1] = fmaf(w, f.y, a[2 * j + 1]);
     }
   } else {
-    const uint32_t x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      acc[2 * j] = fmaf(w, bf16lo(x[j]), acc[2 * j]);
-      acc[2 * j + 1] = fmaf(w, bf16hi(x[j]), acc[2 * j + 1]);
+      a[2 * j] = fmaf(w, bf16lo(x[j]), a[2 * j]);
+      a[2 * j + 1] = fmaf(w, bf16hi(x[j]), a[2 * j + 1]);
     }
   }
+#else
+#if MFET_BAG_ACC == 2
+  if (DT != MFET_F32 && !wsum) {  // acc += x with the 16-bit operand converted inside the add
+    float* a = reinterpret_cast<float*>(acc);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if constexpr (DT == MFET_F16)
+        asm("{.reg .b16 l, h; mov.b32 {l, h}, %2; add.rn.f32.f16 %0, l, %0; add.rn.f32.f16 %1, h, %1;}"
+            : "+f"(a[2 * j]), "+f"(a[2 * j + 1]) : "r"(x[j]));
+      else
+        asm("{.reg .b16 l, h; mov.b32 {l, h}, %2; add.rn.f32.bf16 %0, l, %0; add.rn.f32.bf16 %1, h, %1;}"
+            : "+f"(a[2 * j]), "+f"(a[2 * j + 1]) : "r"(x[j]));
+    }
+    return;
+  }
+#endif
+  const unsigned long long w2 = pack2(__float_as_uint(w), __float_as_uint(w));
+  if constexpr (DT == MFET_F32) {
+    fma2(acc[0], pack2(x[0], x[1]), w2);
+    fma2(acc[1], pack2(x[2], x[3]), w2);
+  } else if constexpr (DT == MFET_F16) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&x[j]));
+      fma2(acc[j], pack2(__float_as_uint(f.x), __float_as_uint(f.y)), w2);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) fma2(acc[j], pack2(x[j] << 16, x[j] & 0xFFFF0000u), w2);
+  }
+#endif
+  (void)wsum;
 }
 
 // Combine the GG row groups of a bag group. While a lane holds more than one
@@ -96,6 +149,16 @@ struct ReduceScatter {
   }
 };
 
+// One bag of a bag group, as the round loop sees it.
+struct BagCur {
+  int64_t lo;   // first ID of the bag
+  int len;      // its length (0 when this group has no bag)
+  int bi;       // index inside the tile
+  int maxlen;   // longest / shortest bag among the warp's bag groups: the warp
+  int minlen;   // runs maxlen rows, the first minlen of them without predicates
+  bool have;
+};
+
 // IND = false: rows come from the slot's table by hashing the ID.
 // IND = true : rows of a host-table slot come from the HBM cache or the staging
 //              buffer, through the dedup inverse map (feat_lo = first ID of the
@@ -108,13 +171,14 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
   constexpr int GG = GL / LPR;          // row groups per bag group
   constexpr int NG = 256 / GL;          // bag groups per block
   constexpr int U = LPR < MFET_BAG_U ? LPR : MFET_BAG_U;  // row loads in flight per lane
-  constexpr int NF = (E / GG) > 0 ? (E / GG) : 1;  // values a lane stores
+  constexpr int NF = (E / GG) > 0 ? (E / GG) : 1;         // values a lane stores
 
   const int lane = threadIdx.x & 31;
   const int gl = lane & (GL - 1);
   const int sub = gl / LPR;
   const int c = gl & (LPR - 1);
   const int grp = threadIdx.x / GL;
+  const bool all_chunks = (int)s.chunks == LPR;  // no idle chunk lanes
   const bool chunk_ok = c < (int)s.chunks;
   const bool wsum = s.pooling == MFET_POOL_WSUM;
   const bool pre = (p.flags & 1u) != 0;
@@ -123,56 +187,98 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
   const uint64_t stride16 = s.stride >> 4;
   const unsigned long long* ids = reinterpret_cast<const unsigned long long*>(p.ids);
 
-  // bags perm[q0 .. q1) of the tile, NG at a time (perm orders the tile by falling length,
-  // so the bag groups of one warp work on bags of similar length)
-  for (int qb = q0; qb < q1; qb += NG) {
+  // bags perm[q0 .. q1) of the tile, NG at a time
+  auto open_bag = [&](int qb, BagCur& b) {
     const int q = qb + grp;
-    const bool have = q < q1;
-    const int bi = have ? (int)perm[q] : 0;
-    int64_t lo = 0;
-    int len = 0;
-    if (have) {
-      lo = soff[bi];
-      int64_t l = soff[bi + 1] - lo;
+    b.have = q < q1;
+    b.bi = b.have ? (int)perm[q] : 0;
+    b.lo = 0;
+    b.len = 0;
+    if (b.have) {
+      b.lo = soff[b.bi];
+      int64_t l = soff[b.bi + 1] - b.lo;
       if (l < 0) {
         if (gl == 0) atomicOr(p.err, (uint32_t)MFET_DEV_OFFSETS);
         l = 0;
       }
-      len = l > 0x7FFFFFFF ? 0x7FFFFFFF : (int)l;
+      b.len = l > 0x7FFFFFFF ? 0x7FFFFFFF : (int)l;
     }
-    const int maxlen = __reduce_max_sync(kFull, len);
+    b.maxlen = __reduce_max_sync(kFull, b.len);
+    b.minlen = __reduce_min_sync(kFull, b.len);
+  };
+  // the ID (or, IND, the row location) and weight of position base+gl of a bag
+  auto fetch = [&](const BagCur& b, int base, uint64_t& id, float& w) {
+    id = 0;
+    w = 1.f;
+    if (base + gl < b.len) {
+      const int64_t i = b.lo + base + gl;
+      if constexpr (IND) id = (uint32_t)__ldg(ip.inverse + (i - feat_lo));
+      else id = __ldcs(ids + i);
+      if (wsum) w = __ldcs(p.weights + i);
+    }
+  };
 
-    float acc[E];
+  if (q0 >= q1) return;
+  BagCur cur;
+  open_bag(q0, cur);
+  int qb = q0, base = 0;
+  uint64_t id_c;
+  float w_c;
+  fetch(cur, 0, id_c, w_c);
+
+  unsigned long long acc[E / 2];
 #pragma unroll
-    for (int j = 0; j < E; ++j) acc[j] = 0.f;
+  for (int j = 0; j < E / 2; ++j) acc[j] = 0ull;
 
-    for (int base = 0; base < maxlen; base += GL) {
-      // every lane of the bag group hashes one ID of this round
-      uint64_t off16 = ~0ULL;  // sentinel: no row
-      float w = 1.f;
-      if (base + gl < len) {
-        const int64_t i = lo + base + gl;
-        if constexpr (IND) {
-          const int32_t j = __ldg(ip.inverse + (i - feat_lo));
-          const int32_t sidx = __ldg(ip.src + j);
-          const uint8_t* rowp = sidx >= 0 ? ip.cache_data + (uint64_t)sidx * ip.row_bytes
-                                          : ip.staging + (uint64_t)(-1 - sidx) * ip.row_bytes;
-          off16 = reinterpret_cast<uint64_t>(rowp) >> 4;
-        } else {
-          const uint64_t id = __ldcs(ids + i);
-          const uint64_t row = pre ? id : mod_rows(splitmix64(id ^ s.seed), s.rows, s.magic);
-          if (row < s.rows) off16 = row * stride16;
-          else atomicOr(p.err, (uint32_t)MFET_DEV_ROW_RANGE);
-        }
-        if (wsum) w = __ldcs(p.weights + i);
+  while (true) {
+    // ---- what comes after this round; its IDs are requested now -------------
+    const bool last_round = base + GL >= cur.maxlen;  // warp-uniform
+    BagCur nxt = cur;
+    int nbase = base + GL, nqb = qb;
+    bool more = true;
+    if (last_round) {
+      nqb = qb + NG;
+      nbase = 0;
+      more = nqb < q1;
+      if (more) open_bag(nqb, nxt);
+    }
+    uint64_t id_n = 0;
+    float w_n = 1.f;
+    if (more) fetch(nxt, nbase, id_n, w_n);
+
+    // ---- this round: every lane of the bag group resolves one row ------------
+    uint64_t off16 = ~0ULL;  // sentinel: no row
+    if (base + gl < cur.len) {
+      if constexpr (IND) {
+        const int32_t sidx = __ldg(ip.src + (uint32_t)id_c);
+        const uint8_t* rowp = sidx >= 0 ? ip.cache_data + (uint64_t)sidx * ip.row_bytes
+                                        : ip.staging + (uint64_t)(-1 - sidx) * ip.row_bytes;
+        off16 = reinterpret_cast<uint64_t>(rowp) >> 4;
+      } else {
+        const uint64_t row = pre ? id_c : mod_rows(splitmix64(id_c ^ s.seed), s.rows, s.magic);
+        if (row < s.rows) off16 = row * stride16;
+        else atomicOr(p.err, (uint32_t)MFET_DEV_ROW_RANGE);
       }
-      const uint32_t off_lo = (uint32_t)off16, off_hi = (uint32_t)(off16 >> 32);
-      const int cnt = min(GL, maxlen - base);  // warp-uniform
+    }
+    const uint32_t off_lo = (uint32_t)off16, off_hi = (uint32_t)(off16 >> 32);
+    const int cnt = min(GL, cur.maxlen - base);                 // IDs of the longest group
+    const int full = all_chunks ? min(GL, cur.minlen - base) : 0;  // IDs that every group has
 #pragma unroll
-      for (int u0 = 0; u0 < LPR; u0 += U) {
-        if (u0 * GG >= cnt) break;
-        uint4 v[U];
-        float wk[U];
+    for (int u0 = 0; u0 < LPR; u0 += U) {
+      if (u0 * GG >= cnt) break;
+      uint4 v[U];
+      float wk[U];
+      if ((u0 + U) * GG <= full && !pre) {
+        // every lane has a row in each of the U steps: no predicates
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+          const int src = (u0 + k) * GG + sub;
+          const uint32_t o_lo = __shfl_sync(kFull, off_lo, src, GL);
+          const uint32_t o_hi = narrow ? 0u : __shfl_sync(kFull, off_hi, src, GL);
+          wk[k] = wsum ? __shfl_sync(kFull, w_c, src, GL) : 1.f;
+          v[k] = ld_row16(tbase + ((((uint64_t)o_hi << 32) | o_lo) << 4));
+        }
+      } else {
 #pragma unroll
         for (int k = 0; k < U; ++k) {
           const int src = (u0 + k) * GG + sub;
@@ -185,43 +291,59 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
             o_hi = __shfl_sync(kFull, off_hi, src, GL);
             valid = (o_lo & o_hi) != 0xFFFFFFFFu;
           }
-          wk[k] = wsum ? __shfl_sync(kFull, w, src, GL) : 1.f;
+          wk[k] = wsum ? __shfl_sync(kFull, w_c, src, GL) : 1.f;
           v[k] = make_uint4(0u, 0u, 0u, 0u);
-          if (valid && chunk_ok)
-            v[k] = ld_row16(tbase + ((((uint64_t)o_hi << 32) | o_lo) << 4));
+          if (valid && chunk_ok) v[k] = ld_row16(tbase + ((((uint64_t)o_hi << 32) | o_lo) << 4));
         }
-#pragma unroll
-        for (int k = 0; k < U; ++k) accumulate<DT>(acc, v[k], wk[k]);
       }
+#pragma unroll
+      for (int k = 0; k < U; ++k) accumulate<DT>(acc, v[k], wk[k], wsum);
     }
 
-    int off = 0;
-    bool writer = have && chunk_ok;
-    ReduceScatter<E, 0, GG, LPR>::run(acc, sub, off, writer);
-    if (s.pooling == MFET_POOL_MEAN && len > 0) {
-      const float fl = (float)len;
+    // ---- end of the bag: combine row groups, scale, store ---------------------
+    if (last_round) {
+      float a[E];
 #pragma unroll
-      for (int j = 0; j < NF; ++j) acc[j] = __fdiv_rn(acc[j], fl);
-    }
-    if (writer) {
-      float* o = p.out + (int64_t)(b0 + bi) * p.out_ld + s.col_off + c * E + off;
-      if (p.flags & 2u) {
-        if constexpr (NF >= 4) {
+      for (int j = 0; j < E / 2; ++j) {
+        a[2 * j] = __uint_as_float((uint32_t)acc[j]);
+        a[2 * j + 1] = __uint_as_float((uint32_t)(acc[j] >> 32));
+        acc[j] = 0ull;
+      }
+      int off = 0;
+      bool writer = cur.have && chunk_ok;
+      ReduceScatter<E, 0, GG, LPR>::run(a, sub, off, writer);
+      if (s.pooling == MFET_POOL_MEAN && cur.len > 0) {
+        const float fl = (float)cur.len;
 #pragma unroll
-          for (int j = 0; j < NF; j += 4)
-            __stcs(reinterpret_cast<float4*>(o + j), make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]));
-        } else if constexpr (NF == 2) {
-          __stcs(reinterpret_cast<float2*>(o), make_float2(acc[0], acc[1]));
+        for (int j = 0; j < NF; ++j) a[j] = __fdiv_rn(a[j], fl);
+      }
+      if (writer) {
+        float* o = p.out + (int64_t)(b0 + cur.bi) * p.out_ld + s.col_off + c * E + off;
+        if (p.flags & 2u) {
+          if constexpr (NF >= 4) {
+#pragma unroll
+            for (int j = 0; j < NF; j += 4)
+              __stcs(reinterpret_cast<float4*>(o + j), make_float4(a[j], a[j + 1], a[j + 2], a[j + 3]));
+          } else if constexpr (NF == 2) {
+            __stcs(reinterpret_cast<float2*>(o), make_float2(a[0], a[1]));
+          } else {
+            __stcs(o, a[0]);
+          }
         } else {
-          __stcs(o, acc[0]);
-        }
-      } else {
 #pragma unroll
-        for (int j = 0; j < NF; ++j) __stcs(o + j, acc[j]);
+          for (int j = 0; j < NF; ++j) __stcs(o + j, a[j]);
+        }
       }
     }
+    if (!more) break;
+    cur = nxt;
+    qb = nqb;
+    base = nbase;
+    id_c = id_n;
+    w_c = w_n;
   }
 }
+
 
 #define MFET_POOL_ARGS p, s, soff, b0, perm, ip, feat_lo
 

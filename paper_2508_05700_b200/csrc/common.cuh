@@ -52,6 +52,9 @@ struct mfet_tables {
   uint64_t launches = 0;
   int32_t group_policy = 0;
   int32_t tile = 0;  // bags per block; 0 = chosen from the batch size
+  int32_t profile = 0;             // 1: time the stages of the host-table path with events
+  cudaEvent_t prof_ev[4] = {nullptr, nullptr, nullptr, nullptr};
+  bool prof_valid = false;
 };
 
 namespace mfet {

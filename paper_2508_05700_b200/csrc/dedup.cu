@@ -78,40 +78,44 @@ __global__ void __launch_bounds__(kSortThreads) hist_kernel(NSrc ns, const uint6
     }
   }
   __syncthreads();
-  hist[(size_t)threadIdx.x * nblk + blockIdx.x] = h[threadIdx.x];
+  hist[(size_t)blockIdx.x * 256 + threadIdx.x] = h[threadIdx.x];  // block-major: coalesced
 }
 
-// Exclusive scan of `total` counters in place, one block. Each thread owns a
-// contiguous segment; segment sums are scanned with shuffles.
-__global__ void __launch_bounds__(1024) scan_counters_kernel(uint32_t* __restrict__ a, int total) {
-  __shared__ uint32_t warp_sum[32];
-  const int per = (total + 1023) / 1024;
-  const int begin = min(total, (int)threadIdx.x * per), end = min(total, begin + per);
+// Turns the per-tile digit counts hist[tile][digit] into the global start position of
+// every (digit, tile) pair in digit-major order: start(d, b) = sum of all counts of smaller
+// digits + counts of digit d in tiles before b. One block of 1024 threads: thread t owns
+// digit t & 255 and a quarter of the tiles, so every load and store is coalesced across
+// the digits and the loads of a thread are independent of each other.
+__global__ void __launch_bounds__(1024) scan_counters_kernel(uint32_t* __restrict__ hist, int nblk) {
+  __shared__ uint32_t part[4][256];
+  __shared__ uint32_t digit_excl[256];
+  __shared__ uint32_t warp_tot[8];
+  const int d = threadIdx.x & 255, q = threadIdx.x >> 8;
+  const int per = (nblk + 3) / 4;
+  const int b0 = min(nblk, q * per), b1 = min(nblk, b0 + per);
   uint32_t sum = 0;
-  for (int i = begin; i < end; ++i) sum += a[i];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t inc = sum;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-    if (lane >= d) inc += t;
-  }
-  if (lane == 31) warp_sum[warp] = inc;
+  for (int b = b0; b < b1; ++b) sum += hist[(size_t)b * 256 + d];
+  part[q][d] = sum;
   __syncthreads();
-  if (warp == 0) {
-    uint32_t w = warp_sum[lane];
+  if (threadIdx.x < 256) {  // exclusive scan of the 256 digit totals
+    const uint32_t tot = part[0][d] + part[1][d] + part[2][d] + part[3][d];
+    const int lane = threadIdx.x & 31;
+    uint32_t inc = tot;
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, w, d);
-      if (lane >= d) w += t;
+    for (int k = 1; k < 32; k <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, k);
+      if (lane >= k) inc += t;
     }
-    warp_sum[lane] = w;
+    digit_excl[d] = inc - tot;
+    if (lane == 31) warp_tot[threadIdx.x >> 5] = inc;
   }
   __syncthreads();
-  uint32_t run = inc - sum + (warp ? warp_sum[warp - 1] : 0u);
-  for (int i = begin; i < end; ++i) {
-    const uint32_t v = a[i];
-    a[i] = run;
+  uint32_t run = digit_excl[d];
+  for (int w = 0; w < (d >> 5); ++w) run += warp_tot[w];
+  for (int qq = 0; qq < q; ++qq) run += part[qq][d];
+  for (int b = b0; b < b1; ++b) {
+    const uint32_t v = hist[(size_t)b * 256 + d];
+    hist[(size_t)b * 256 + d] = run;
     run += v;
   }
 }
@@ -129,7 +133,7 @@ __global__ void __launch_bounds__(kSortThreads) scatter_kernel(NSrc ns, const ui
   int64_t lo;
   const int64_t n = resolve_n(ns, &lo);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  base[threadIdx.x] = hist[(size_t)threadIdx.x * nblk + blockIdx.x];
+  base[threadIdx.x] = hist[(size_t)blockIdx.x * 256 + threadIdx.x];
 #pragma unroll
   for (int w = 0; w < kSortThreads / 32; ++w) wcnt[w][threadIdx.x] = 0;
   __syncthreads();
@@ -417,7 +421,7 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
                                                       a.hash->magic, a.hash->pre_hashed, shift, hist, nblk, a.err);
     else
       hist_kernel<false><<<nblk, kSortThreads, 0, s>>>(a.ns, kin, nullptr, nullptr, 0, 0, 0, 0, shift, hist, nblk, a.err);
-    scan_counters_kernel<<<1, 1024, 0, s>>>(hist, 256 * nblk);
+    scan_counters_kernel<<<1, 1024, 0, s>>>(hist, nblk);
     scatter_kernel<<<nblk, kSortThreads, 0, s>>>(a.ns, kin, iin, kout, iout, shift, hist, nblk);
     *launches += 3;
     // next pass reads what this one wrote

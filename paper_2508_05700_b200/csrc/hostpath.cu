@@ -111,12 +111,16 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
   a.miss_rows = (int64_t*)(ws + L.miss_rows);
   a.n_miss = counters + 1;
   a.err = t->err_dev;
+  const bool prof = t->profile != 0;
+  if (prof) cudaEventRecord(t->prof_ev[0], side);
   if (launch_dedup(a, &t->launches, side) != cudaSuccess) return MFET_ERR_CUDA;
+  if (prof) cudaEventRecord(t->prof_ev[1], side);
 
   const uint32_t chunks = (uint32_t)(tb.row_bytes / 16);
   if (launch_fetch(tb.dev_ptr, tb.stride, chunks, a.miss_rows, a.n_miss, 0, ws + L.staging, side) != cudaSuccess)
     return MFET_ERR_CUDA;
   t->launches += 1;
+  if (prof) cudaEventRecord(t->prof_ev[2], side);
 
   IndirectParams ip{a.inverse, a.src, tb.cache.data, ws + L.staging, tb.row_bytes, t->ws_max_ids};
   BagParams p = base;
@@ -145,6 +149,10 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
       t->launches += 1;
       n = 0;
     }
+  }
+  if (prof) {
+    cudaEventRecord(t->prof_ev[3], side);
+    t->prof_valid = true;
   }
   return MFET_OK;
 }

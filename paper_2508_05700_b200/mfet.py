@@ -23,6 +23,7 @@ LOC_DEVICE, LOC_HOST = 0, 1
 VAL_NORMAL, VAL_GRID = 0, 1
 OPT_GROUP_POLICY = 1
 OPT_TILE = 2
+OPT_PROFILE = 3
 OK = 0
 ERR_INVALID_ARG, ERR_NOT_REGISTERED, ERR_ALIGNMENT, ERR_UNSUPPORTED_DIM = -1, -2, -3, -4
 ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
@@ -33,7 +34,7 @@ EXPORTS = [
     "mfet_hash_ids", "mfet_embedding_bag_forward", "mfet_dedup_rows", "mfet_cache_bytes",
     "mfet_cache_build", "mfet_workspace_bytes", "mfet_set_workspace", "mfet_host_io_bytes",
     "mfet_embedding_bag_forward_host", "mfet_table_fill", "mfet_query_status", "mfet_set_option",
-    "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static",
+    "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static", "mfet_profile_read",
 ]
 STATIC_DEDUP_MAX_IDS = 262144
 
@@ -77,6 +78,7 @@ _lib.mfet_table_fill.argtypes = [_P, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uin
                                  C.c_uint32, _P]
 _lib.mfet_query_status.argtypes = [_P, C.POINTER(C.c_uint32), C.c_int32]
 _lib.mfet_set_option.argtypes = [_P, C.c_int32, C.c_int64]
+_lib.mfet_profile_read.argtypes = [_P, C.POINTER(C.c_float)]
 _lib.mfet_launch_count.argtypes = [_P, C.POINTER(C.c_uint64)]
 for _n in EXPORTS:
     if _n not in ("mfet_row_bytes", "mfet_status_string"):
@@ -218,6 +220,13 @@ def mfet_query_status(h, clear: bool = False) -> int:
 
 def mfet_set_option(h, option: int, value: int) -> None:
     _check(_lib.mfet_set_option(h, option, value), "mfet_set_option")
+
+
+def mfet_profile_read(h):
+    """(dedup_ms, fetch_ms, pool_ms) of the last forward call's host-table path."""
+    ms = (C.c_float * 3)()
+    _check(_lib.mfet_profile_read(h, ms), "mfet_profile_read")
+    return tuple(float(x) for x in ms)
 
 
 def mfet_launch_count(h) -> int:
