@@ -262,6 +262,12 @@ MFET_API int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value);
  * call's host-table path to finish. Needs MFET_OPT_PROFILE = 1 (else INVALID_ARG). */
 MFET_API int mfet_profile_read(mfet_tables_t* t, float* stage_ms /*host float[3]*/);
 
+/* Distinct rows (n_unique) and distinct rows not found in the HBM cache (n_miss: what
+ * crossed PCIe) of the most recent host-table slot that ran. Waits for the internal
+ * stream and copies two counters out of the workspace. Errors: INVALID_ARG, WORKSPACE
+ * (no workspace attached), CUDA. */
+MFET_API int mfet_host_path_counts(mfet_tables_t* t, int64_t* n_unique /*host*/, int64_t* n_miss /*host*/);
+
 /* Number of kernels the library has launched on behalf of this handle. */
 MFET_API int mfet_launch_count(const mfet_tables_t* t, uint64_t* launches /*host*/);
 

@@ -252,6 +252,13 @@ int mfet_set_workspace(mfet_tables_t* t, void* dev_ptr, uint64_t bytes, int64_t 
   int rc = mfet_workspace_bytes(t, max_ids, &need);
   if (rc != MFET_OK) return rc;
   if (bytes < need) return MFET_ERR_WORKSPACE;
+  {
+    // the arrival counters inside the workspace must start at zero (kernels leave them at zero)
+    WsLayout L;
+    workspace_layout(max_ids, 16, &L);
+    DeviceGuard g(t->device);
+    if (!g.ok || cudaMemset(static_cast<uint8_t*>(dev_ptr) + L.counters, 0, 64) != cudaSuccess) return MFET_ERR_CUDA;
+  }
   t->ws = dev_ptr;
   t->ws_bytes = bytes;
   t->ws_max_ids = max_ids;

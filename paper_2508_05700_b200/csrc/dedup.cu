@@ -38,15 +38,55 @@ __device__ __forceinline__ int64_t resolve_n(const NSrc& s, int64_t* lo) {
 
 // ---- pass kernels --------------------------------------------------------
 
-// Digit histogram of one tile. With HASH the keys are produced here from the
-// raw IDs (first pass of a host-table slot) and stored for the later passes.
+// True in exactly one block of the grid: the one whose arrival is the last. That block may
+// then read what all other blocks wrote before they arrived. Nobody waits for anybody.
+__device__ __forceinline__ bool last_block_arrives(uint32_t* ticket) {
+  __shared__ bool last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (last) __threadfence();
+  return last;
+}
+
+// Turns the per-tile digit counts hist[tile][digit] into the global start position of every
+// (digit, tile) pair in digit-major order: start(d, b) = all counts of smaller digits + counts
+// of digit d in tiles before b. Run by the 256 threads of one block; thread d owns digit d, so
+// loads and stores are coalesced across the digits and a thread's loads are independent.
+__device__ __forceinline__ void scan_digit_counts(uint32_t* hist, int nblk) {
+  __shared__ uint32_t warp_tot[8];
+  const int d = threadIdx.x;
+  uint32_t tot = 0;
+  for (int b = 0; b < nblk; ++b) tot += __ldcg(hist + (size_t)b * 256 + d);
+  const int lane = d & 31;
+  uint32_t inc = tot;
+#pragma unroll
+  for (int k = 1; k < 32; k <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, k);
+    if (lane >= k) inc += t;
+  }
+  if (lane == 31) warp_tot[d >> 5] = inc;
+  __syncthreads();
+  uint32_t run = inc - tot;
+  for (int w = 0; w < (d >> 5); ++w) run += warp_tot[w];
+  for (int b = 0; b < nblk; ++b) {
+    const uint32_t v = __ldcg(hist + (size_t)b * 256 + d);
+    hist[(size_t)b * 256 + d] = run;
+    run += v;
+  }
+}
+
+// Digit histogram of one tile; the block that finishes last turns all histograms into
+// scatter positions. With HASH the keys are produced here from the raw IDs (first pass of
+// a host-table slot) and stored for the later passes.
 template <bool HASH>
 __global__ void __launch_bounds__(kSortThreads) hist_kernel(NSrc ns, const uint64_t* __restrict__ keys_in,
                                                             uint64_t* __restrict__ keys_store,
                                                             const uint64_t* __restrict__ ids, uint64_t seed,
                                                             uint64_t rows, uint64_t magic, uint32_t pre_hashed,
-                                                            int shift, uint32_t* __restrict__ hist, int nblk,
-                                                            uint32_t* err) {
+                                                            int shift, uint32_t* hist, int nblk,
+                                                            uint32_t* err, uint32_t* ticket) {
   __shared__ uint32_t h[256];
   int64_t lo;
   const int64_t n = resolve_n(ns, &lo);
@@ -58,11 +98,13 @@ __global__ void __launch_bounds__(kSortThreads) hist_kernel(NSrc ns, const uint6
   h[threadIdx.x] = 0;
   __syncthreads();
   const int64_t base = (int64_t)blockIdx.x * kSortTile;
+  const int lane = threadIdx.x & 31;
 #pragma unroll
   for (int r = 0; r < kSortRounds; ++r) {
     const int64_t i = base + r * kSortThreads + threadIdx.x;
-    if (i < n) {
-      uint64_t k;
+    const bool valid = i < n;
+    uint64_t k = 0;
+    if (valid) {
       if (HASH) {
         const uint64_t id = __ldcs(reinterpret_cast<const unsigned long long*>(ids) + lo + i);
         k = pre_hashed ? id : mod_rows(splitmix64(id ^ seed), rows, magic);
@@ -74,49 +116,18 @@ __global__ void __launch_bounds__(kSortThreads) hist_kernel(NSrc ns, const uint6
       } else {
         k = keys_in[i];
       }
-      atomicAdd(&h[(k >> shift) & 255u], 1u);
     }
+    // one shared-memory add per distinct digit of the warp: Zipf heads repeat the same row
+    // thousands of times, and per-thread adds on one counter would serialise
+    const uint32_t d = (uint32_t)(k >> shift) & 255u;
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, valid ? d : 256u + (uint32_t)lane);
+    if (valid && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&h[d], (uint32_t)__popc(peers));
   }
   __syncthreads();
   hist[(size_t)blockIdx.x * 256 + threadIdx.x] = h[threadIdx.x];  // block-major: coalesced
-}
-
-// Turns the per-tile digit counts hist[tile][digit] into the global start position of
-// every (digit, tile) pair in digit-major order: start(d, b) = sum of all counts of smaller
-// digits + counts of digit d in tiles before b. One block of 1024 threads: thread t owns
-// digit t & 255 and a quarter of the tiles, so every load and store is coalesced across
-// the digits and the loads of a thread are independent of each other.
-__global__ void __launch_bounds__(1024) scan_counters_kernel(uint32_t* __restrict__ hist, int nblk) {
-  __shared__ uint32_t part[4][256];
-  __shared__ uint32_t digit_excl[256];
-  __shared__ uint32_t warp_tot[8];
-  const int d = threadIdx.x & 255, q = threadIdx.x >> 8;
-  const int per = (nblk + 3) / 4;
-  const int b0 = min(nblk, q * per), b1 = min(nblk, b0 + per);
-  uint32_t sum = 0;
-  for (int b = b0; b < b1; ++b) sum += hist[(size_t)b * 256 + d];
-  part[q][d] = sum;
-  __syncthreads();
-  if (threadIdx.x < 256) {  // exclusive scan of the 256 digit totals
-    const uint32_t tot = part[0][d] + part[1][d] + part[2][d] + part[3][d];
-    const int lane = threadIdx.x & 31;
-    uint32_t inc = tot;
-#pragma unroll
-    for (int k = 1; k < 32; k <<= 1) {
-      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, k);
-      if (lane >= k) inc += t;
-    }
-    digit_excl[d] = inc - tot;
-    if (lane == 31) warp_tot[threadIdx.x >> 5] = inc;
-  }
-  __syncthreads();
-  uint32_t run = digit_excl[d];
-  for (int w = 0; w < (d >> 5); ++w) run += warp_tot[w];
-  for (int qq = 0; qq < q; ++qq) run += part[qq][d];
-  for (int b = b0; b < b1; ++b) {
-    const uint32_t v = hist[(size_t)b * 256 + d];
-    hist[(size_t)b * 256 + d] = run;
-    run += v;
+  if (last_block_arrives(ticket)) {
+    scan_digit_counts(hist, nblk);
+    if (threadIdx.x == 0) *ticket = 0;  // ready for the next pass
   }
 }
 
@@ -218,7 +229,9 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* total,
 template <bool PROBE>
 __global__ void __launch_bounds__(kScanThreads) unique_count_kernel(NSrc ns, const uint64_t* __restrict__ keys,
                                                                     CacheDev cache, int32_t* __restrict__ probe_tmp,
-                                                                    uint32_t* __restrict__ tile_counts, int nblk) {
+                                                                    uint32_t* tile_counts, int nblk, uint32_t* ticket,
+                                                                    int64_t* __restrict__ n_unique,
+                                                                    int64_t* __restrict__ n_miss) {
   __shared__ uint32_t sh[8];
   int64_t lo;
   const int64_t n = resolve_n(ns, &lo);
@@ -247,52 +260,29 @@ __global__ void __launch_bounds__(kScanThreads) unique_count_kernel(NSrc ns, con
     tile_counts[blockIdx.x] = th;
     if (PROBE) tile_counts[nblk + blockIdx.x] = tm;
   }
-}
-
-// Pass 2 (one block): exclusive scan of the per-tile counts; totals out.
-__global__ void __launch_bounds__(1024) unique_scan_kernel(uint32_t* __restrict__ tile_counts, int nblk, int n_arrays,
-                                                           int64_t* __restrict__ n_unique, int64_t* __restrict__ n_miss) {
-  __shared__ uint32_t warp_sum[32];
-  for (int a = 0; a < n_arrays; ++a) {
-    uint32_t* arr = tile_counts + (size_t)a * nblk;
-    const int per = (nblk + 1023) / 1024;
-    const int begin = min(nblk, (int)threadIdx.x * per), end = min(nblk, begin + per);
-    uint32_t sum = 0;
-    for (int i = begin; i < end; ++i) sum += arr[i];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t inc = sum;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-      if (lane >= d) inc += t;
-    }
-    __syncthreads();
-    if (lane == 31) warp_sum[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t w = warp_sum[lane];
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, w, d);
-        if (lane >= d) w += t;
+  // the block that finishes last scans the per-tile counts and publishes the totals
+  if (last_block_arrives(ticket)) {
+    for (int a = 0; a < (PROBE ? 2 : 1); ++a) {
+      uint32_t* arr = tile_counts + (size_t)a * nblk;
+      uint32_t run = 0;
+      for (int i0 = 0; i0 < nblk; i0 += kScanThreads) {
+        const int i = i0 + threadIdx.x;
+        const uint32_t v = i < nblk ? __ldcg(arr + i) : 0u;
+        uint32_t tot;
+        const uint32_t ex = block_excl_scan(v, &tot, sh);
+        if (i < nblk) arr[i] = run + ex;
+        run += tot;
       }
-      warp_sum[lane] = w;
+      if (threadIdx.x == 0) {
+        if (a == 0) *n_unique = (int64_t)run;
+        else *n_miss = (int64_t)run;
+      }
     }
-    __syncthreads();
-    uint32_t run = inc - sum + (warp ? warp_sum[warp - 1] : 0u);
-    for (int i = begin; i < end; ++i) {
-      const uint32_t v = arr[i];
-      arr[i] = run;
-      run += v;
-    }
-    if (threadIdx.x == 1023) {
-      if (a == 0) *n_unique = (int64_t)run;
-      else *n_miss = (int64_t)run;
-    }
+    if (threadIdx.x == 0) *ticket = 0;
   }
 }
 
-// Pass 3: write uniq, inverse and (PROBE) the per-unique source and the list of
+// Pass 2: write uniq, inverse and (PROBE) the per-unique source and the list of
 // missed rows.
 template <bool PROBE>
 __global__ void __launch_bounds__(kScanThreads) unique_write_kernel(NSrc ns, const uint64_t* __restrict__ keys,
@@ -402,6 +392,7 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
   uint32_t* ib = (uint32_t*)(ws + L.idx_b);
   uint32_t* hist = (uint32_t*)(ws + L.hist);
   uint32_t* tile_counts = (uint32_t*)(ws + L.tile_counts);
+  uint32_t* tickets = (uint32_t*)(ws + L.counters + 32);  // two arrival counters, zero between launches
 
   const int64_t cap = a.ns.offsets ? a.ns.cap : a.ns.n_imm;
   const int nblk = (int)((cap + kSortTile - 1) / kSortTile) > 0 ? (int)((cap + kSortTile - 1) / kSortTile) : 1;
@@ -418,12 +409,11 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
     const int shift = 8 * p;
     if (p == 0 && a.hash)
       hist_kernel<true><<<nblk, kSortThreads, 0, s>>>(a.ns, nullptr, ka, a.hash->ids, a.hash->seed, a.hash->rows,
-                                                      a.hash->magic, a.hash->pre_hashed, shift, hist, nblk, a.err);
+                                                      a.hash->magic, a.hash->pre_hashed, shift, hist, nblk, a.err, tickets);
     else
-      hist_kernel<false><<<nblk, kSortThreads, 0, s>>>(a.ns, kin, nullptr, nullptr, 0, 0, 0, 0, shift, hist, nblk, a.err);
-    scan_counters_kernel<<<1, 1024, 0, s>>>(hist, nblk);
+      hist_kernel<false><<<nblk, kSortThreads, 0, s>>>(a.ns, kin, nullptr, nullptr, 0, 0, 0, 0, shift, hist, nblk, a.err, tickets);
     scatter_kernel<<<nblk, kSortThreads, 0, s>>>(a.ns, kin, iin, kout, iout, shift, hist, nblk);
-    *launches += 3;
+    *launches += 2;
     // next pass reads what this one wrote
     kin = kout;
     iin = iout;
@@ -433,18 +423,18 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
   // kin / iin: sorted keys and their original positions; iout is free
   int32_t* probe_tmp = (int32_t*)iout;
   if (a.cache) {
-    unique_count_kernel<true><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, *a.cache, probe_tmp, tile_counts, nblk2);
-    unique_scan_kernel<<<1, 1024, 0, s>>>(tile_counts, nblk2, 2, a.n_unique, a.n_miss);
+    unique_count_kernel<true><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, *a.cache, probe_tmp, tile_counts, nblk2,
+                                                             tickets + 1, a.n_unique, a.n_miss);
     unique_write_kernel<true><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, iin, probe_tmp, tile_counts, nblk2, a.uniq,
                                                             a.inverse, a.src, a.miss_rows);
   } else {
     CacheDev none{};
-    unique_count_kernel<false><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, none, nullptr, tile_counts, nblk2);
-    unique_scan_kernel<<<1, 1024, 0, s>>>(tile_counts, nblk2, 1, a.n_unique, nullptr);
+    unique_count_kernel<false><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, none, nullptr, tile_counts, nblk2, tickets + 1,
+                                                              a.n_unique, nullptr);
     unique_write_kernel<false><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, iin, nullptr, tile_counts, nblk2, a.uniq,
                                                              a.inverse, nullptr, nullptr);
   }
-  *launches += 3;
+  *launches += 2;
   return cudaGetLastError();
 }
 
@@ -468,7 +458,8 @@ constexpr uint64_t kOffIdxA = kOffKeysB + pad256(kStaticMaxIds * 8);
 constexpr uint64_t kOffIdxB = kOffIdxA + pad256(kStaticMaxIds * 4);
 constexpr uint64_t kOffHist = kOffIdxB + pad256(kStaticMaxIds * 4);
 constexpr uint64_t kOffTiles = kOffHist + pad256(kStaticSortBlocks * 256 * 4);
-constexpr uint64_t kStaticScratchBytes = kOffTiles + pad256(kStaticScanBlocks * 2 * 4);
+constexpr uint64_t kOffCounters = kOffTiles + pad256(kStaticScanBlocks * 2 * 4);
+constexpr uint64_t kStaticScratchBytes = kOffCounters + 256;
 
 // In host code this name is only a handle of the symbol, not a device address:
 // the address is asked from the runtime once per device (below).
@@ -529,6 +520,7 @@ extern "C" int mfet_dedup_rows_static(int32_t device, const int64_t* rows, int64
       a.layout.idx_b = kOffIdxB;
       a.layout.hist = kOffHist;
       a.layout.tile_counts = kOffTiles;
+      a.layout.counters = kOffCounters;
       a.uniq = uniq;
       a.inverse = inverse;
       a.n_unique = n_unique;

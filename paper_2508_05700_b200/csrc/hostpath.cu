@@ -194,6 +194,24 @@ int mfet_dedup_rows(mfet_tables_t* t, const int64_t* rows, int64_t n, int64_t* u
   return rc;
 }
 
+int mfet_host_path_counts(mfet_tables_t* t, int64_t* n_unique, int64_t* n_miss) {
+  if (!t || !n_unique || !n_miss) return MFET_ERR_INVALID_ARG;
+  if (!t->ws) return MFET_ERR_WORKSPACE;
+  WsLayout L;
+  workspace_layout(t->ws_max_ids, 16, &L);
+  int prev = 0;
+  if (cudaGetDevice(&prev) != cudaSuccess) return MFET_ERR_CUDA;
+  if (prev != t->device && cudaSetDevice(t->device) != cudaSuccess) return MFET_ERR_CUDA;
+  int64_t c[2] = {0, 0};
+  bool ok = cudaStreamSynchronize(t->side) == cudaSuccess &&
+            cudaMemcpy(c, static_cast<uint8_t*>(t->ws) + L.counters, sizeof(c), cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (prev != t->device) cudaSetDevice(prev);
+  if (!ok) return MFET_ERR_CUDA;
+  *n_unique = c[0];
+  *n_miss = c[1];
+  return MFET_OK;
+}
+
 int mfet_cache_bytes(const mfet_tables_t* t, int32_t table_id, int64_t n, uint64_t* bytes) {
   if (!t || !bytes || n < 0 || table_id < 0 || table_id >= (int32_t)t->tables.size()) return MFET_ERR_INVALID_ARG;
   const TableHost& tb = t->tables[(size_t)table_id];

@@ -34,7 +34,7 @@ EXPORTS = [
     "mfet_hash_ids", "mfet_embedding_bag_forward", "mfet_dedup_rows", "mfet_cache_bytes",
     "mfet_cache_build", "mfet_workspace_bytes", "mfet_set_workspace", "mfet_host_io_bytes",
     "mfet_embedding_bag_forward_host", "mfet_table_fill", "mfet_query_status", "mfet_set_option",
-    "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static", "mfet_profile_read",
+    "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static", "mfet_profile_read", "mfet_host_path_counts",
 ]
 STATIC_DEDUP_MAX_IDS = 262144
 
@@ -79,6 +79,7 @@ _lib.mfet_table_fill.argtypes = [_P, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uin
 _lib.mfet_query_status.argtypes = [_P, C.POINTER(C.c_uint32), C.c_int32]
 _lib.mfet_set_option.argtypes = [_P, C.c_int32, C.c_int64]
 _lib.mfet_profile_read.argtypes = [_P, C.POINTER(C.c_float)]
+_lib.mfet_host_path_counts.argtypes = [_P, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
 _lib.mfet_launch_count.argtypes = [_P, C.POINTER(C.c_uint64)]
 for _n in EXPORTS:
     if _n not in ("mfet_row_bytes", "mfet_status_string"):
@@ -227,6 +228,13 @@ def mfet_profile_read(h):
     ms = (C.c_float * 3)()
     _check(_lib.mfet_profile_read(h, ms), "mfet_profile_read")
     return tuple(float(x) for x in ms)
+
+
+def mfet_host_path_counts(h):
+    """(distinct rows, distinct rows missing from the cache) of the last host-table slot."""
+    a, b = C.c_int64(), C.c_int64()
+    _check(_lib.mfet_host_path_counts(h, C.byref(a), C.byref(b)), "mfet_host_path_counts")
+    return int(a.value), int(b.value)
 
 
 def mfet_launch_count(h) -> int:
