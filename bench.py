@@ -59,6 +59,8 @@ def algorithmic_bytes(w: gi.Workload, b: gi.Batch, slots=None) -> int:
 
 
 def gi_row_bytes(t: gi.TableSpec) -> int:
+    if t.dtype == gi.INT4:
+        return (t.dim // 2 + 4 + 15) // 16 * 16
     return t.dim * (4 if t.dtype == gi.F32 else 2)
 
 

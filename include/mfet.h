@@ -76,7 +76,7 @@ typedef struct {
                            is supplied later by mfet_host_tables_register).            */
   uint64_t rows;        /* 1 .. 2^63-1                                                  */
   uint32_t dim;         /* elements per row; stored row bytes must be a multiple of 16  */
-  uint32_t dtype;       /* MFET_F32 / MFET_F16 / MFET_BF16 (MFET_INT4 is reserved: rejected)   */
+  uint32_t dtype;       /* MFET_F32 / MFET_F16 / MFET_BF16 / MFET_INT4 (dim % 8 == 0)          */
   uint32_t location;    /* MFET_LOC_DEVICE / MFET_LOC_HOST                              */
   uint32_t flags;       /* must be 0                                                    */
   uint64_t hash_seed;   /* XORed into the raw ID before hashing; 0 = plain hash         */
@@ -236,7 +236,13 @@ MFET_API int mfet_embedding_bag_forward_host(mfet_tables_t* t, const mfet_batch_
  *   MFET_VAL_NORMAL: s = sum of the four 16-bit fields of u;
  *                    v = float(s - 131070) * fp32(0.01 / 37837.227)
  *   MFET_VAL_GRID:   v = float((u & 255) - 128) * 2^-13
- * rounded to nearest-even into `dtype` (F32 / F16 / BF16).
+ * rounded to nearest-even into `dtype` (F32 / F16 / BF16). MFET_INT4 (paper, Section
+ * 4.1.2: the tables are post-training quantised to INT4; the paper gives no format, this
+ * is the library's): per row, scale = fp16((max-min)/15), bias = fp16(min), code =
+ * clamp(rint((v - bias)/scale), 0, 15) with the quotient in double precision; stored as
+ * dim/2 bytes of codes (element d in the low nibble of byte d/2 when d is even), the fp16
+ * scale, the fp16 bias, zero padding to a multiple of 16 bytes. A looked-up element is
+ * fma(code, scale, bias) in fp32.
  * data: dev memory, or pinned+mapped host memory (written through the unified
  * address space); rows [row0, row0+n_rows) are written. */
 MFET_API int mfet_table_fill(void* data, uint64_t row0, uint64_t n_rows, uint32_t dim, uint32_t dtype,

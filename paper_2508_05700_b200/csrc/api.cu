@@ -61,7 +61,8 @@ int mfet_tables_create(const mfet_table_desc_t* descs, int32_t n_tables, int32_t
   for (int32_t i = 0; i < n_tables; ++i) {
     const mfet_table_desc_t& d = descs[i];
     if (d.rows == 0 || d.rows >= (1ULL << 63) || d.dim == 0 || d.flags != 0) return MFET_ERR_INVALID_ARG;
-    if (d.dtype > MFET_BF16 || d.location > MFET_LOC_HOST) return MFET_ERR_INVALID_ARG;
+    if (d.dtype > MFET_INT4 || d.location > MFET_LOC_HOST) return MFET_ERR_INVALID_ARG;
+    if (d.dtype == MFET_INT4 && (d.dim % 8u) != 0) return MFET_ERR_UNSUPPORTED_DIM;
     const uint64_t rb = mfet_row_bytes(d.dim, d.dtype);
     if (rb == 0 || rb % 16 != 0) return MFET_ERR_UNSUPPORTED_DIM;
     const uint64_t stride = d.row_stride_bytes ? d.row_stride_bytes : rb;
@@ -171,7 +172,8 @@ int mfet_hash_ids(const mfet_tables_t* t, int32_t table_id, const uint64_t* ids,
 int mfet_table_fill(void* data, uint64_t row0, uint64_t n_rows, uint32_t dim, uint32_t dtype,
                     uint64_t row_stride_bytes, uint64_t value_key, uint32_t value_mode,
                     mfet_stream_t stream) {
-  if (!data || dim == 0 || dtype > MFET_BF16 || value_mode > MFET_VAL_GRID) return MFET_ERR_INVALID_ARG;
+  if (!data || dim == 0 || dtype > MFET_INT4 || value_mode > MFET_VAL_GRID) return MFET_ERR_INVALID_ARG;
+  if (dtype == MFET_INT4 && (dim % 8u) != 0) return MFET_ERR_UNSUPPORTED_DIM;
   const uint64_t rb = mfet_row_bytes(dim, dtype);
   if (rb == 0 || rb % 16 != 0) return MFET_ERR_UNSUPPORTED_DIM;
   const uint64_t stride = row_stride_bytes ? row_stride_bytes : rb;
@@ -341,7 +343,10 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
       if (rc != MFET_OK) return rc;
     } else {
       // rows wider than 512 bytes are covered by several entries of <= 32 chunks
-      const uint32_t chunks_total = (uint32_t)(tb.row_bytes / 16);
+      // a lane's chunk: 16 bytes, or 4 bytes of codes for INT4 rows
+      const bool int4 = tb.desc.dtype == MFET_INT4;
+      const uint32_t chunk_bytes = int4 ? 4u : 16u;
+      const uint32_t chunks_total = int4 ? tb.desc.dim / 8u : (uint32_t)(tb.row_bytes / 16);
       const uint32_t epc = tb.desc.dtype == MFET_F32 ? 4u : 8u;  // elements per chunk
       for (uint32_t c0 = 0; c0 < chunks_total; c0 += 32) {
         if (n == kMaxSlotsPerLaunch) {
@@ -350,7 +355,8 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
         }
         SlotDev& sd = p.slot[n++];
         const uint32_t ch = chunks_total - c0 < 32 ? chunks_total - c0 : 32;
-        sd.table = tb.dev_ptr + (uint64_t)c0 * 16;
+        sd.table = tb.dev_ptr + (uint64_t)c0 * chunk_bytes;
+        sd.meta_off = int4 ? tb.desc.dim / 2u - c0 * chunk_bytes : 0u;
         sd.rows = tb.desc.rows;
         sd.magic = tb.magic;
         sd.seed = tb.desc.hash_seed;

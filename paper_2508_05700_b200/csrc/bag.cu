@@ -47,10 +47,19 @@ namespace {
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kLongBag = MFET_BAG_LONG;  // bags at least this long get a whole warp
 
+// A lane's piece of a row: 16 bytes (4 fp32 or 8 fp16/bf16 values), or for INT4 rows
+// 4 bytes (8 four-bit codes) plus the row's fp16 scale/bias pair.
 template <int DT>
 struct ChunkElems {
   static constexpr int value = (DT == MFET_F32) ? 4 : 8;
+  static constexpr int bytes = (DT == MFET_INT4) ? 4 : 16;
 };
+
+template <int DT>
+__device__ __forceinline__ uint4 load_chunk(const uint8_t* chunk, const uint8_t* meta) {
+  if constexpr (DT == MFET_INT4) return make_uint4(ld_row4(chunk), ld_row4(meta), 0u, 0u);
+  else return ld_row16(chunk);
+}
 
 __device__ __forceinline__ unsigned long long pack2(uint32_t lo, uint32_t hi) {
   unsigned long long r;
@@ -67,6 +76,24 @@ __device__ __forceinline__ void fma2(unsigned long long& a, unsigned long long x
 // fp32). The up-conversion of fp16 / bf16 is exact.
 template <int DT>
 __device__ __forceinline__ void accumulate(unsigned long long* acc, const uint4& v, float w, bool wsum) {
+  if constexpr (DT == MFET_INT4) {
+    // value = fma(code, scale, bias) in fp32 (one rounding), then acc += w * value
+    const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+    const unsigned long long s2 = pack2(__float_as_uint(sb.x), __float_as_uint(sb.x));
+    const unsigned long long b2 = pack2(__float_as_uint(sb.y), __float_as_uint(sb.y));
+    const unsigned long long w2 = pack2(__float_as_uint(w), __float_as_uint(w));
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      // codes 2j, 2j+1 -> exact floats through the 2^23 mantissa trick
+      const uint32_t lo = 0x4B000000u | ((v.x >> (8 * j)) & 15u), hi = 0x4B000000u | ((v.x >> (8 * j + 4)) & 15u);
+      const float c0 = __uint_as_float(lo) - 8388608.f, c1 = __uint_as_float(hi) - 8388608.f;
+      unsigned long long val = b2;
+      fma2(val, pack2(__float_as_uint(c0), __float_as_uint(c1)), s2);
+      fma2(acc[j], val, w2);
+    }
+    (void)wsum;
+    return;
+  }
   const uint32_t x[4] = {v.x, v.y, v.z, v.w};
 #if MFET_BAG_ACC == 0
   float* a = reinterpret_cast<float*>(acc);
@@ -183,7 +210,8 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
   const bool wsum = s.pooling == MFET_POOL_WSUM;
   const bool pre = (p.flags & 1u) != 0;
   const bool narrow = !IND && s.narrow != 0;
-  const uint8_t* tbase = s.table + c * 16;  // IND: s.table = byte offset of the column block
+  const uint8_t* tbase = s.table + c * ChunkElems<DT>::bytes;  // IND: s.table = byte offset of the column block
+  const uint8_t* mbase = s.table + s.meta_off;               // INT4: the row's scale/bias pair
   const uint64_t stride16 = s.stride >> 4;
   const unsigned long long* ids = reinterpret_cast<const unsigned long long*>(p.ids);
 
@@ -276,7 +304,8 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
           const uint32_t o_lo = __shfl_sync(kFull, off_lo, src, GL);
           const uint32_t o_hi = narrow ? 0u : __shfl_sync(kFull, off_hi, src, GL);
           wk[k] = wsum ? __shfl_sync(kFull, w_c, src, GL) : 1.f;
-          v[k] = ld_row16(tbase + ((((uint64_t)o_hi << 32) | o_lo) << 4));
+          const uint64_t ro = (((uint64_t)o_hi << 32) | o_lo) << 4;
+          v[k] = load_chunk<DT>(tbase + ro, mbase + ro);
         }
       } else {
 #pragma unroll
@@ -293,7 +322,8 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
           }
           wk[k] = wsum ? __shfl_sync(kFull, w_c, src, GL) : 1.f;
           v[k] = make_uint4(0u, 0u, 0u, 0u);
-          if (valid && chunk_ok) v[k] = ld_row16(tbase + ((((uint64_t)o_hi << 32) | o_lo) << 4));
+          const uint64_t ro = (((uint64_t)o_hi << 32) | o_lo) << 4;
+          if (valid && chunk_ok) v[k] = load_chunk<DT>(tbase + ro, mbase + ro);
         }
       }
 #pragma unroll
@@ -373,7 +403,9 @@ __device__ __forceinline__ void pool_tile_dt(const BagParams& p, const SlotDev& 
   }
 }
 
-template <bool IND>
+// Q4 = true: the build of the kernel that also decodes INT4 rows (kept apart so that the
+// common kernels stay small).
+template <bool IND, bool Q4>
 __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParams& ip) {
   __shared__ int64_t soff[kMaxTile + 1];
   __shared__ int64_t sfeat[2];
@@ -430,6 +462,12 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   if (p.group_policy == 1) n_long = 0;
   if (p.group_policy == 2) n_long = nb;
 
+  if constexpr (Q4) {
+    if (s.dtype == MFET_INT4) {
+      pool_tile_dt<MFET_INT4, IND>(MFET_POOL_ARGS, n_long, nb);
+      return;
+    }
+  }
   switch (s.dtype) {
     case MFET_F32: pool_tile_dt<MFET_F32, IND>(MFET_POOL_ARGS, n_long, nb); break;
     case MFET_F16: pool_tile_dt<MFET_F16, IND>(MFET_POOL_ARGS, n_long, nb); break;
@@ -439,27 +477,45 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
 
 __global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_kernel(const __grid_constant__ BagParams p) {
   const IndirectParams none{};
-  bag_body<false>(p, none);
+  bag_body<false, false>(p, none);
+}
+
+__global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_q4_kernel(const __grid_constant__ BagParams p) {
+  const IndirectParams none{};
+  bag_body<false, true>(p, none);
 }
 
 __global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_indirect_kernel(const __grid_constant__ BagParams p,
                                                            const __grid_constant__ IndirectParams ip) {
-  bag_body<true>(p, ip);
+  bag_body<true, false>(p, ip);
+}
+
+__global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_indirect_q4_kernel(const __grid_constant__ BagParams p,
+                                                              const __grid_constant__ IndirectParams ip) {
+  bag_body<true, true>(p, ip);
 }
 
 }  // namespace
 
+static bool any_int4(const BagParams& p) {
+  for (int i = 0; i < p.n_slots; ++i)
+    if (p.slot[i].dtype == MFET_INT4) return true;
+  return false;
+}
+
 cudaError_t launch_bag_indirect(const BagParams& p, const IndirectParams& ip, cudaStream_t s) {
   const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
   if (blocks == 0) return cudaSuccess;
-  bag_indirect_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, ip);
+  if (any_int4(p)) bag_indirect_q4_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, ip);
+  else bag_indirect_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, ip);
   return cudaGetLastError();
 }
 
 cudaError_t launch_bag(const BagParams& p, cudaStream_t s) {
   const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
   if (blocks == 0) return cudaSuccess;
-  bag_kernel<<<(unsigned)blocks, 256, 0, s>>>(p);
+  if (any_int4(p)) bag_q4_kernel<<<(unsigned)blocks, 256, 0, s>>>(p);
+  else bag_kernel<<<(unsigned)blocks, 256, 0, s>>>(p);
   return cudaGetLastError();
 }
 

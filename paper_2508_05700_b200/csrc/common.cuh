@@ -77,7 +77,7 @@ struct SlotDev {
   uint8_t lpr_log2;      // lanes per row = 1 << lpr_log2 >= chunks
   uint8_t narrow;        // 1: (rows*stride)/16 fits 32 bits
   uint16_t pad;
-  uint32_t pad2;
+  uint32_t meta_off;     // INT4: byte offset of the row's fp16 scale/bias pair from `table`
 };
 static_assert(sizeof(SlotDev) == 64, "SlotDev must stay 64 bytes");
 
@@ -131,6 +131,12 @@ __device__ __forceinline__ uint4 ld_row16(const void* p) {
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ uint32_t ld_row4(const void* p) {
+  uint32_t v;
+  asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
   return v;
 }
 

@@ -76,9 +76,52 @@ __global__ void __launch_bounds__(256) fill_kernel(uint8_t* __restrict__ data, u
   }
 }
 
+// INT4 rows (one thread per row; not a hot kernel): the row's fp32 values are generated,
+// scale = fp16((max-min)/15) and bias = fp16(min) are fixed, every value becomes the code
+// clamp(rint((x - bias) / scale), 0, 15) - the quotient in double precision, so that every
+// implementation of this definition rounds the same way -, two codes per byte, low nibble
+// first, then scale and bias, then zero padding up to a multiple of 16 bytes.
+__global__ void __launch_bounds__(128) fill_int4_kernel(uint8_t* __restrict__ data, uint64_t row0, uint64_t n_rows,
+                                                        uint32_t dim, uint64_t stride, uint64_t row_bytes,
+                                                        uint64_t key, uint32_t mode) {
+  const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_rows) return;
+  const uint64_t r = row0 + i;
+  float lo = table_value(key, mode, r * dim), hi = lo;
+  for (uint32_t d = 1; d < dim; ++d) {
+    const float x = table_value(key, mode, r * dim + d);
+    lo = fminf(lo, x);
+    hi = fmaxf(hi, x);
+  }
+  const __half sh = __float2half_rn(__fdiv_rn(__fsub_rn(hi, lo), 15.0f)), bh = __float2half_rn(lo);
+  const double scale = (double)__half2float(sh), bias = (double)__half2float(bh);
+  uint8_t* row = data + r * stride;
+  for (uint32_t d = 0; d < dim; d += 8) {
+    uint32_t word = 0;
+    for (uint32_t j = 0; j < 8; ++j) {
+      int code = 0;
+      if (scale > 0.0) {
+        const double q = rint(((double)table_value(key, mode, r * dim + d + j) - bias) / scale);
+        code = (int)fmin(15.0, fmax(0.0, q));
+      }
+      word |= (uint32_t)code << (4 * j);
+    }
+    *reinterpret_cast<uint32_t*>(row + d / 2) = word;
+  }
+  *reinterpret_cast<uint32_t*>(row + dim / 2) = (uint32_t)__half_as_ushort(sh) | ((uint32_t)__half_as_ushort(bh) << 16);
+  for (uint64_t b = dim / 2 + 4; b < row_bytes; b += 4) *reinterpret_cast<uint32_t*>(row + b) = 0u;
+}
+
 cudaError_t launch_fill(void* data, uint64_t row0, uint64_t n_rows, uint32_t dim, uint32_t dtype,
                         uint64_t stride, uint64_t key, uint32_t mode, cudaStream_t s) {
   if (n_rows == 0) return cudaSuccess;
+  if (dtype == MFET_INT4) {
+    const uint64_t blocks = (n_rows + 127) / 128;
+    if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    fill_int4_kernel<<<(unsigned)blocks, 128, 0, s>>>((uint8_t*)data, row0, n_rows, dim, stride,
+                                                      mfet_row_bytes(dim, dtype), key, mode);
+    return cudaGetLastError();
+  }
   const uint32_t chunks = (uint32_t)(mfet_row_bytes(dim, dtype) / 16);
   uint64_t total = n_rows * chunks;
   uint64_t blocks = (total + 255) / 256;

@@ -127,12 +127,16 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
   p.flags &= ~1u;  // the indirect path never hashes
   p.flags |= base.flags & 2u;
   const uint32_t epc = tb.desc.dtype == MFET_F32 ? 4u : 8u;
+  const bool int4 = tb.desc.dtype == MFET_INT4;
+  const uint32_t chunk_bytes = int4 ? 4u : 16u;
+  const uint32_t pool_chunks = int4 ? tb.desc.dim / 8u : chunks;  // a lane's chunk: 16 bytes, INT4: 4 bytes of codes
   int n = 0;
-  for (uint32_t c0 = 0; c0 < chunks; c0 += 32) {
+  for (uint32_t c0 = 0; c0 < pool_chunks; c0 += 32) {
     SlotDev& sd = p.slot[n++];
     std::memset(&sd, 0, sizeof(sd));
-    const uint32_t ch = chunks - c0 < 32 ? chunks - c0 : 32;
-    sd.table = reinterpret_cast<const uint8_t*>((uintptr_t)c0 * 16);  // byte offset inside the row
+    const uint32_t ch = pool_chunks - c0 < 32 ? pool_chunks - c0 : 32;
+    sd.table = reinterpret_cast<const uint8_t*>((uintptr_t)c0 * chunk_bytes);  // byte offset inside the row
+    sd.meta_off = int4 ? tb.desc.dim / 2u - c0 * chunk_bytes : 0u;
     sd.rows = tb.desc.rows;
     sd.stride = tb.row_bytes;
     sd.feature = (uint32_t)feature;
@@ -143,7 +147,7 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
     uint8_t lg = 1;
     while ((1u << lg) < ch) ++lg;
     sd.lpr_log2 = lg;
-    if (n == kMaxSlotsPerLaunch || c0 + 32 >= chunks) {
+    if (n == kMaxSlotsPerLaunch || c0 + 32 >= pool_chunks) {
       p.n_slots = n;
       if (launch_bag_indirect(p, ip, side) != cudaSuccess) return MFET_ERR_CUDA;
       t->launches += 1;

@@ -513,3 +513,57 @@ def test_device_error_bits_for_bad_prehashed_rows_and_offsets():
         assert not out2.cpu().numpy()[1].any()
     finally:
         mt.close()
+
+
+# ------------------------------------------------------------------- INT4 ---
+
+@pytest.mark.parametrize("dim", [8, 24, 32, 64, 128, 264])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_int4_table_fill_bit_exact(dim, mode):
+    """Paper, Section 4.1.2 (INT4 post-training quantisation; the row format is this library's)."""
+    m = mfet()
+    rows, key = 1237, 0x0F1E2D3C4B5A6978
+    rb = m.row_bytes(dim, m.INT4)
+    assert rb % 16 == 0 and rb >= dim // 2 + 4
+    buf = torch.full((rows * rb,), 0xAB, dtype=torch.uint8, device="cuda")
+    m.mfet_table_fill(buf, 0, rows, dim, m.INT4, 0, key, mode, _stream())
+    got = buf.cpu().numpy().reshape(rows, rb)
+    want = orc.table_fill(orc.Table(rows=rows, dim=dim, dtype=orc.INT4, value_key=key, value_mode=mode))
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("dim", [8, 24, 32, 64, 128, 264])
+@pytest.mark.parametrize("policy", [0, 1, 2])
+def test_int4_pooling_parity(dim, policy):
+    specs = [gi.TableSpec(5003, dim, gi.INT4, 0x1234567, 0xABCDEF0123), gi.TableSpec(977, dim, gi.INT4, 99, 777)]
+    rng = np.random.default_rng(dim + policy)
+    with DeviceTables(specs) as dt:
+        dt.m.mfet_set_option(dt.h, dt.m.OPT_GROUP_POLICY, policy)
+        B, F = 61, 2
+        off = _ragged(rng, F * B, "mixed")
+        ids = rng.integers(0, 2**40, size=int(off[-1]), dtype=np.uint64)
+        w = rng.random(ids.size).astype(np.float32)
+        sf, ti, po = [0, 0, 1, 1], [0, 1, 1, 0], [0, 2, 1, 2]
+        got = forward(dt, B, F, sf, ti, po, ids, off, w)
+        ref = orc.embedding_bag(dt.oracle_tables, B, F, sf, ti, po, ids, off, w)
+        assert_close(got, ref, "int4 dim %d" % dim)
+        # single-ID bags return the decoded row itself, bit for bit
+        one = forward(dt, 8, 1, [0], [0], [0], np.arange(8, dtype=np.uint64), np.arange(9, dtype=np.int64), None,
+                      ids_are_rows=True)
+        want = np.stack([orc.decode_row(dt.oracle_tables[0], r) for r in range(8)])
+        assert np.array_equal(one, want)
+
+
+def test_int4_host_table_behind_the_cache():
+    """The quantised table in host memory (the paper's serving set-up: INT4 tables on the CPU side)."""
+    w = gi.make_workload(5, rows_scale=0.001, batch_scale=0.125)
+    w.tables[0].dtype = gi.INT4
+    b = gi.make_batch(w, 0)
+    n_host = int(b.offsets[w.batch] - b.offsets[0])
+    with DeviceTables(w.tables) as dt:
+        dt.set_workspace(n_host + 1024)
+        ref = workload_oracle(dt, w, b)
+        cold = workload_forward(dt, w, b)
+        assert_close(cold, ref, "int4 host table, no cache")
+        dt.build_cache(0, _hot_rows(dt, w, 0, 0, int(w.tables[0].rows * 0.05), w.tables[0].rows))
+        assert np.array_equal(workload_forward(dt, w, b), cold)
