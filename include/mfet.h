@@ -47,6 +47,7 @@ enum { MFET_F32 = 0, MFET_F16 = 1, MFET_BF16 = 2, MFET_INT4 = 3 };
 enum { MFET_POOL_SUM = 0, MFET_POOL_MEAN = 1, MFET_POOL_WSUM = 2 };
 enum { MFET_LOC_DEVICE = 0, MFET_LOC_HOST = 1 };
 enum { MFET_VAL_NORMAL = 0, MFET_VAL_GRID = 1 };
+enum { MFET_BATCH_IDS_ARE_ROWS = 1, MFET_BATCH_PREFETCHED = 2 }; /* mfet_batch_shape_t.flags */
 enum { MFET_OPT_GROUP_POLICY = 1, MFET_OPT_TILE = 2, MFET_OPT_PROFILE = 3 };
 
 enum {
@@ -88,7 +89,8 @@ typedef struct {
   int32_t batch;               /* B >= 0                                              */
   int32_t n_features;          /* F >= 1                                              */
   int32_t n_slots;             /* L >= 1                                              */
-  int32_t flags;               /* bit0: `ids` already hold row indices (no hashing)   */
+  int32_t flags;               /* MFET_BATCH_IDS_ARE_ROWS: `ids` already hold row indices (no
+                                  hashing); MFET_BATCH_PREFETCHED: see mfet_host_prefetch */
   const int32_t* slot_feature; /* host int32[L]: feature read by each slot            */
   int64_t out_ld;              /* floats per row of `out`; 0 = sum of the slots' dims */
 } mfet_batch_shape_t;
@@ -154,6 +156,22 @@ MFET_API int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape
                                const uint64_t* ids, const int64_t* offsets, const float* weights,
                                const int32_t* table_ids, const int32_t* pooling, float* out,
                                mfet_stream_t stream);
+
+/* Early fetch for the next batch (paper, Sections 1 and 3.4: the embedding fetch from the
+ * CPU side is started as early as possible so that it runs in parallel with the rest of
+ * serving and adds no latency). For a batch with exactly ONE host-table slot this runs that
+ * slot's hash -> dedup -> cache probe -> fetch of the missed rows now, on the library's
+ * internal stream (ordered after what `stream` holds at the call, not joined back to it),
+ * into one of two result sets of the workspace. The matching mfet_embedding_bag_forward
+ * call - same ids/offsets contents, shape.flags | MFET_BATCH_PREFETCHED - then only pools,
+ * and gives the same bits as a call without prefetch. At most two prefetches may be
+ * outstanding; they are consumed in order. ids/offsets must stay unchanged until the
+ * matching forward call has been issued. A forward call without the flag for a batch that
+ * has a host-table slot is refused (INVALID_ARG) while a prefetch is outstanding.
+ * Errors: INVALID_ARG (not exactly one host-table slot, two prefetches outstanding, ...),
+ * NOT_REGISTERED, WORKSPACE, ALIGNMENT, CUDA. */
+MFET_API int mfet_host_prefetch(mfet_tables_t* t, const mfet_batch_shape_t* shape, const uint64_t* ids,
+                       const int64_t* offsets, const int32_t* table_ids, mfet_stream_t stream);
 
 /* In-batch dedup of hashed rows, done before host reads so that each distinct
  * row crosses PCIe once (paper, Section 3.3 motivates keeping host traffic off
@@ -273,6 +291,14 @@ MFET_API int mfet_profile_read(mfet_tables_t* t, float* stage_ms /*host float[3]
  * stream and copies two counters out of the workspace. Errors: INVALID_ARG, WORKSPACE
  * (no workspace attached), CUDA. */
 MFET_API int mfet_host_path_counts(mfet_tables_t* t, int64_t* n_unique /*host*/, int64_t* n_miss /*host*/);
+
+/* Version tag of a table set (paper, Section 3.3 and Algorithm 2: embeddings travel with the
+ * version id of the tables that produced them, so that they are scored by the matching
+ * upper model). The library stores the tag and returns it unchanged; the caller sends it
+ * along with `out`. Two table sets with different tags can be alive side by side during a
+ * roll-out (Algorithm 1). Default tag: 0. */
+MFET_API int mfet_tables_set_version(mfet_tables_t* t, uint64_t version);
+MFET_API int mfet_tables_version(const mfet_tables_t* t, uint64_t* version /*host*/);
 
 /* Number of kernels the library has launched on behalf of this handle. */
 MFET_API int mfet_launch_count(const mfet_tables_t* t, uint64_t* launches /*host*/);

@@ -191,6 +191,18 @@ int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits, int32_t cle
   return MFET_OK;
 }
 
+int mfet_tables_set_version(mfet_tables_t* t, uint64_t version) {
+  if (!t) return MFET_ERR_INVALID_ARG;
+  t->version = version;
+  return MFET_OK;
+}
+
+int mfet_tables_version(const mfet_tables_t* t, uint64_t* version) {
+  if (!t || !version) return MFET_ERR_INVALID_ARG;
+  *version = t->version;
+  return MFET_OK;
+}
+
 int mfet_launch_count(const mfet_tables_t* t, uint64_t* launches) {
   if (!t || !launches) return MFET_ERR_INVALID_ARG;
   *launches = t->launches;
@@ -267,17 +279,60 @@ int mfet_set_workspace(mfet_tables_t* t, void* dev_ptr, uint64_t bytes, int64_t 
   return MFET_OK;
 }
 
+int mfet_host_prefetch(mfet_tables_t* t, const mfet_batch_shape_t* shape, const uint64_t* ids,
+                       const int64_t* offsets, const int32_t* table_ids, mfet_stream_t stream_) {
+  if (!t || !shape || !table_ids || !shape->slot_feature || !ids || !offsets) return MFET_ERR_INVALID_ARG;
+  const int32_t B = shape->batch, F = shape->n_features, L = shape->n_slots;
+  if (B < 1 || F < 1 || L < 1 || (shape->flags & ~3)) return MFET_ERR_INVALID_ARG;
+  int host_slot = -1, n_host = 0;
+  for (int32_t s = 0; s < L; ++s) {
+    const int32_t ti = table_ids[s], f = shape->slot_feature[s];
+    if (ti < 0 || ti >= (int32_t)t->tables.size() || f < 0 || f >= F) return MFET_ERR_INVALID_ARG;
+    const TableHost& tb = t->tables[(size_t)ti];
+    if (!tb.registered) return MFET_ERR_NOT_REGISTERED;
+    if (tb.desc.location == MFET_LOC_HOST) {
+      host_slot = s;
+      ++n_host;
+    }
+  }
+  if (n_host != 1) return MFET_ERR_INVALID_ARG;
+  if (!t->ws || t->ws_max_ids <= 0) return MFET_ERR_WORKSPACE;
+  if (t->prefetched - t->consumed >= 2) return MFET_ERR_INVALID_ARG;  // both result sets are taken
+  if ((reinterpret_cast<uintptr_t>(ids) & 7u) || (reinterpret_cast<uintptr_t>(offsets) & 7u)) return MFET_ERR_ALIGNMENT;
+  DeviceGuard g(t->device);
+  if (!g.ok) return MFET_ERR_CUDA;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  BagParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.ids = ids;
+  p.offsets = offsets;
+  p.err = t->err_dev;
+  p.batch = B;
+  p.flags = (uint32_t)(shape->flags & 1);
+  // the internal stream starts after what `stream` holds now (the batch's inputs) and is not joined back
+  if (cudaEventRecord(t->ev_fork, stream) != cudaSuccess) return MFET_ERR_CUDA;
+  if (cudaStreamWaitEvent(t->side, t->ev_fork, 0) != cudaSuccess) return MFET_ERR_CUDA;
+  const TableHost& tb = t->tables[(size_t)table_ids[host_slot]];
+  int rc = run_host_slot(t, tb, p, shape->slot_feature[host_slot], MFET_POOL_SUM, 0, t->side, 1,
+                         (int)(t->prefetched & 1u));
+  if (rc != MFET_OK) return rc;
+  t->prefetched += 1;
+  return MFET_OK;
+}
+
 int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape, const uint64_t* ids,
                                const int64_t* offsets, const float* weights, const int32_t* table_ids,
                                const int32_t* pooling, float* out, mfet_stream_t stream_) {
   if (!t || !shape || !table_ids || !pooling || !shape->slot_feature) return MFET_ERR_INVALID_ARG;
   const int32_t B = shape->batch, F = shape->n_features, L = shape->n_slots;
-  if (B < 0 || F < 1 || L < 1 || (shape->flags & ~1)) return MFET_ERR_INVALID_ARG;
+  if (B < 0 || F < 1 || L < 1 || (shape->flags & ~3)) return MFET_ERR_INVALID_ARG;
+  const bool use_prefetch = (shape->flags & MFET_BATCH_PREFETCHED) != 0;
   cudaStream_t stream = (cudaStream_t)stream_;
 
   // validate slots, lay out the output columns
   int64_t total_dim = 0;
   bool any_wsum = false, any_host = false;
+  int n_host_slots = 0;
   for (int32_t s = 0; s < L; ++s) {
     const int32_t ti = table_ids[s], f = shape->slot_feature[s];
     if (ti < 0 || ti >= (int32_t)t->tables.size() || f < 0 || f >= F) return MFET_ERR_INVALID_ARG;
@@ -286,6 +341,7 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
     if (!tb.registered) return MFET_ERR_NOT_REGISTERED;
     any_wsum |= pooling[s] == MFET_POOL_WSUM;
     any_host |= tb.desc.location == MFET_LOC_HOST;
+    n_host_slots += tb.desc.location == MFET_LOC_HOST;
     total_dim += tb.desc.dim;
   }
   const int64_t out_ld = shape->out_ld ? shape->out_ld : total_dim;
@@ -294,6 +350,10 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
   if (!ids || !offsets || !out) return MFET_ERR_INVALID_ARG;
   if (any_wsum && !weights) return MFET_ERR_INVALID_ARG;
   if (any_host && (!t->ws || t->ws_max_ids <= 0)) return MFET_ERR_WORKSPACE;
+  // a prefetched batch has exactly one host-table slot and an unconsumed prefetch; a plain
+  // batch with a host-table slot must not cut in between a prefetch and its forward
+  if (use_prefetch && (n_host_slots != 1 || t->consumed >= t->prefetched)) return MFET_ERR_INVALID_ARG;
+  if (!use_prefetch && any_host && t->consumed != t->prefetched) return MFET_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(ids) & 7u) || (reinterpret_cast<uintptr_t>(offsets) & 7u) ||
       (reinterpret_cast<uintptr_t>(out) & 3u) || (reinterpret_cast<uintptr_t>(weights) & 3u))
     return MFET_ERR_ALIGNMENT;
@@ -339,8 +399,10 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
         if (cudaStreamWaitEvent(t->side, t->ev_fork, 0) != cudaSuccess) return MFET_ERR_CUDA;
         forked = true;
       }
-      int rc = run_host_slot(t, tb, p, shape->slot_feature[s], pooling[s], (uint32_t)col, t->side);
+      int rc = run_host_slot(t, tb, p, shape->slot_feature[s], pooling[s], (uint32_t)col, t->side,
+                             use_prefetch ? 2 : 3, (int)((use_prefetch ? t->consumed : t->prefetched) & 1u));
       if (rc != MFET_OK) return rc;
+      if (use_prefetch) t->consumed += 1;
     } else {
       // rows wider than 512 bytes are covered by several entries of <= 32 chunks
       // a lane's chunk: 16 bytes, or 4 bytes of codes for INT4 rows

@@ -51,6 +51,8 @@ struct mfet_tables {
   int64_t ws_max_ids = 0;
   uint64_t launches = 0;
   int32_t group_policy = 0;
+  uint64_t version = 0;  // caller's tag of this table set (model version)
+  uint64_t prefetched = 0, consumed = 0;  // batches handed to mfet_host_prefetch / pooled from a prefetch
   int32_t tile = 0;  // bags per block; 0 = chosen from the batch size
   int32_t profile = 0;             // 1: time the stages of the host-table path with events
   cudaEvent_t prof_ev[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -166,6 +168,7 @@ struct CacheDev {
 struct WsLayout {
   uint64_t keys_a, keys_b, idx_a, idx_b, hist, tile_counts, counters, uniq, inverse, src, miss_rows,
       staging, total;
+  uint64_t inverse2, src2, staging2;  // second result set: a prefetched batch waits here
   int nblk_sort, nblk_scan;
 };
 
@@ -213,8 +216,9 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
 cudaError_t launch_fetch(const uint8_t* table, uint64_t stride, uint32_t chunks, const int64_t* rows_list,
                          const int64_t* n_ptr, int64_t n_imm, uint8_t* dst, cudaStream_t s);
 cudaError_t launch_bag_indirect(const BagParams& p, const IndirectParams& ip, cudaStream_t s);
+// stage bit0: hash + dedup + probe + fetch into result set `set`; bit1: pool from it
 int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, int32_t feature, int32_t pooling,
-                  uint32_t col, cudaStream_t side);
+                  uint32_t col, cudaStream_t side, int stage, int set);
 
 // launch helpers implemented in the kernel files
 cudaError_t launch_hash(const uint64_t* ids, int64_t n, uint64_t seed, uint64_t rows, uint64_t magic,

@@ -373,6 +373,9 @@ uint64_t workspace_layout(int64_t max_ids, uint64_t max_row_bytes, WsLayout* L) 
   l.src = take(n * 4);
   l.miss_rows = take(n * 8);
   l.staging = take(n * max_row_bytes);
+  l.inverse2 = take(n * 4);
+  l.src2 = take(n * 4);
+  l.staging2 = take(n * max_row_bytes);
   l.total = off;
   if (L) *L = l;
   return off;

@@ -87,7 +87,7 @@ void cache_layout(uint64_t rows, int64_t n, uint64_t row_bytes, CacheLayout* L) 
 }
 
 int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, int32_t feature, int32_t pooling,
-                  uint32_t col, cudaStream_t side) {
+                  uint32_t col, cudaStream_t side, int stage, int set) {
   WsLayout L;
   const uint64_t need = workspace_layout(t->ws_max_ids, tb.row_bytes, &L);
   if (need > t->ws_bytes) return MFET_ERR_WORKSPACE;
@@ -105,24 +105,27 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
   a.layout = L;
   a.cache = &cd;
   a.uniq = (int64_t*)(ws + L.uniq);
-  a.inverse = (int32_t*)(ws + L.inverse);
+  a.inverse = (int32_t*)(ws + (set ? L.inverse2 : L.inverse));
   a.n_unique = counters;
-  a.src = (int32_t*)(ws + L.src);
+  a.src = (int32_t*)(ws + (set ? L.src2 : L.src));
+  uint8_t* staging = ws + (set ? L.staging2 : L.staging);
   a.miss_rows = (int64_t*)(ws + L.miss_rows);
   a.n_miss = counters + 1;
   a.err = t->err_dev;
-  const bool prof = t->profile != 0;
-  if (prof) cudaEventRecord(t->prof_ev[0], side);
-  if (launch_dedup(a, &t->launches, side) != cudaSuccess) return MFET_ERR_CUDA;
-  if (prof) cudaEventRecord(t->prof_ev[1], side);
-
+  const bool prof = t->profile != 0 && stage == 3;
   const uint32_t chunks = (uint32_t)(tb.row_bytes / 16);
-  if (launch_fetch(tb.dev_ptr, tb.stride, chunks, a.miss_rows, a.n_miss, 0, ws + L.staging, side) != cudaSuccess)
-    return MFET_ERR_CUDA;
-  t->launches += 1;
-  if (prof) cudaEventRecord(t->prof_ev[2], side);
+  if (prof) cudaEventRecord(t->prof_ev[0], side);
+  if (stage & 1) {
+    if (launch_dedup(a, &t->launches, side) != cudaSuccess) return MFET_ERR_CUDA;
+    if (prof) cudaEventRecord(t->prof_ev[1], side);
+    if (launch_fetch(tb.dev_ptr, tb.stride, chunks, a.miss_rows, a.n_miss, 0, staging, side) != cudaSuccess)
+      return MFET_ERR_CUDA;
+    t->launches += 1;
+    if (prof) cudaEventRecord(t->prof_ev[2], side);
+  }
+  if (!(stage & 2)) return MFET_OK;
 
-  IndirectParams ip{a.inverse, a.src, tb.cache.data, ws + L.staging, tb.row_bytes, t->ws_max_ids};
+  IndirectParams ip{a.inverse, a.src, tb.cache.data, staging, tb.row_bytes, t->ws_max_ids};
   BagParams p = base;
   p.flags &= ~1u;  // the indirect path never hashes
   p.flags |= base.flags & 2u;

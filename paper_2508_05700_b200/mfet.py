@@ -34,8 +34,10 @@ EXPORTS = [
     "mfet_hash_ids", "mfet_embedding_bag_forward", "mfet_dedup_rows", "mfet_cache_bytes",
     "mfet_cache_build", "mfet_workspace_bytes", "mfet_set_workspace", "mfet_host_io_bytes",
     "mfet_embedding_bag_forward_host", "mfet_table_fill", "mfet_query_status", "mfet_set_option",
-    "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static", "mfet_profile_read", "mfet_host_path_counts",
+    "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static", "mfet_profile_read", "mfet_host_path_counts", "mfet_tables_set_version", "mfet_tables_version",
+    "mfet_host_prefetch",
 ]
+BATCH_IDS_ARE_ROWS, BATCH_PREFETCHED = 1, 2
 STATIC_DEDUP_MAX_IDS = 262144
 
 
@@ -80,6 +82,9 @@ _lib.mfet_query_status.argtypes = [_P, C.POINTER(C.c_uint32), C.c_int32]
 _lib.mfet_set_option.argtypes = [_P, C.c_int32, C.c_int64]
 _lib.mfet_profile_read.argtypes = [_P, C.POINTER(C.c_float)]
 _lib.mfet_host_path_counts.argtypes = [_P, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+_lib.mfet_tables_set_version.argtypes = [_P, C.c_uint64]
+_lib.mfet_tables_version.argtypes = [_P, C.POINTER(C.c_uint64)]
+_lib.mfet_host_prefetch.argtypes = [_P, C.POINTER(BatchShape), _P, _P, _P, _P]
 _lib.mfet_launch_count.argtypes = [_P, C.POINTER(C.c_uint64)]
 for _n in EXPORTS:
     if _n not in ("mfet_row_bytes", "mfet_status_string"):
@@ -235,6 +240,22 @@ def mfet_host_path_counts(h):
     a, b = C.c_int64(), C.c_int64()
     _check(_lib.mfet_host_path_counts(h, C.byref(a), C.byref(b)), "mfet_host_path_counts")
     return int(a.value), int(b.value)
+
+
+def mfet_tables_set_version(h, version: int) -> None:
+    _check(_lib.mfet_tables_set_version(h, version & (2**64 - 1)), "mfet_tables_set_version")
+
+
+def mfet_tables_version(h) -> int:
+    v = C.c_uint64()
+    _check(_lib.mfet_tables_version(h, C.byref(v)), "mfet_tables_version")
+    return int(v.value)
+
+
+def mfet_host_prefetch(h, shape: BatchShape, ids, offsets, table_ids, stream=None) -> None:
+    ti = _i32(table_ids)
+    _check(_lib.mfet_host_prefetch(h, C.byref(shape), _ptr(ids), _ptr(offsets), ti.ctypes.data, _ptr(stream)),
+           "mfet_host_prefetch")
 
 
 def mfet_launch_count(h) -> int:

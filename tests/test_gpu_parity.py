@@ -567,3 +567,79 @@ def test_int4_host_table_behind_the_cache():
         assert_close(cold, ref, "int4 host table, no cache")
         dt.build_cache(0, _hot_rows(dt, w, 0, 0, int(w.tables[0].rows * 0.05), w.tables[0].rows))
         assert np.array_equal(workload_forward(dt, w, b), cold)
+
+
+# ------------------------------------------------- early fetch, version tag --
+
+def test_prefetched_batches_give_the_same_bits_as_the_serial_path():
+    """Paper, Section 3.4: the embedding fetch starts early and overlaps other work; the result
+    must not depend on it."""
+    m = mfet()
+    w = gi.make_workload(5, rows_scale=0.001, batch_scale=0.125)
+    bs = [gi.make_batch(w, j) for j in range(3)]
+    cap = max(int(b.offsets[w.batch] - b.offsets[0]) for b in bs) + 1024
+    with DeviceTables(w.tables) as dt:
+        dt.set_workspace(cap)
+        dt.build_cache(0, _hot_rows(dt, w, 0, 0, int(w.tables[0].rows * 0.02), w.tables[0].rows))
+        serial = [workload_forward(dt, w, b) for b in bs]
+        d_ids = [torch.from_numpy(b.ids.view(np.int64)).cuda() for b in bs]
+        d_off = [torch.from_numpy(b.offsets).cuda() for b in bs]
+        outs = [torch.full((w.batch, w.out_dim), float("nan"), device="cuda") for _ in bs]
+        plain, keep = m.make_shape(w.batch, w.n_features, w.slot_feature)
+        pre, keep2 = m.make_shape(w.batch, w.n_features, w.slot_feature)
+        pre.flags |= m.BATCH_PREFETCHED
+        s = _stream()
+
+        def status(fn, *a):
+            try:
+                fn(*a)
+            except m.MfetError as e:
+                return e.status
+            return 0
+
+        # a flagged forward without a prefetch is refused
+        assert status(m.mfet_embedding_bag_forward, dt.h, pre, d_ids[0], d_off[0], None, w.table_ids, w.pooling,
+                      outs[0], s) == m.ERR_INVALID_ARG
+        m.mfet_host_prefetch(dt.h, plain, d_ids[0], d_off[0], w.table_ids, s)
+        m.mfet_host_prefetch(dt.h, plain, d_ids[1], d_off[1], w.table_ids, s)
+        # both result sets are taken; and an unflagged forward may not cut in
+        assert status(m.mfet_host_prefetch, dt.h, plain, d_ids[2], d_off[2], w.table_ids, s) == m.ERR_INVALID_ARG
+        assert status(m.mfet_embedding_bag_forward, dt.h, plain, d_ids[0], d_off[0], None, w.table_ids, w.pooling,
+                      outs[0], s) == m.ERR_INVALID_ARG
+        m.mfet_embedding_bag_forward(dt.h, pre, d_ids[0], d_off[0], None, w.table_ids, w.pooling, outs[0], s)
+        m.mfet_host_prefetch(dt.h, plain, d_ids[2], d_off[2], w.table_ids, s)
+        m.mfet_embedding_bag_forward(dt.h, pre, d_ids[1], d_off[1], None, w.table_ids, w.pooling, outs[1], s)
+        m.mfet_embedding_bag_forward(dt.h, pre, d_ids[2], d_off[2], None, w.table_ids, w.pooling, outs[2], s)
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(dt.h) == 0
+        for j in range(3):
+            assert np.array_equal(outs[j].cpu().numpy(), serial[j]), j
+        # afterwards the serial path works again
+        assert np.array_equal(workload_forward(dt, w, bs[0]), serial[0])
+    # a batch without exactly one host-table slot cannot be prefetched
+    w2 = gi.make_workload(2, rows_scale=0.001, batch_scale=1 / 16)
+    with DeviceTables(w2.tables) as dt2:
+        b = gi.make_batch(w2, 0)
+        sh, k = m.make_shape(w2.batch, w2.n_features, w2.slot_feature)
+        try:
+            m.mfet_host_prefetch(dt2.h, sh, torch.from_numpy(b.ids.view(np.int64)).cuda(),
+                                 torch.from_numpy(b.offsets).cuda(), w2.table_ids)
+            raise AssertionError("expected INVALID_ARG")
+        except m.MfetError as e:
+            assert e.status == m.ERR_INVALID_ARG
+
+
+def test_version_tag_is_echoed_unchanged():
+    """Paper, Algorithm 2: embeddings are returned together with the version of the tables."""
+    m = mfet()
+    dummy = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    a = m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), 4, 4, m.F32, m.LOC_DEVICE, 0, 0, 0)])
+    b = m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), 4, 4, m.F32, m.LOC_DEVICE, 0, 0, 0)])
+    try:
+        assert m.mfet_tables_version(a) == 0
+        m.mfet_tables_set_version(a, 20250807)
+        m.mfet_tables_set_version(b, 2**64 - 1)
+        assert m.mfet_tables_version(a) == 20250807 and m.mfet_tables_version(b) == 2**64 - 1
+    finally:
+        m.mfet_tables_destroy(a)
+        m.mfet_tables_destroy(b)
