@@ -173,6 +173,23 @@ MFET_API int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape
 MFET_API int mfet_host_prefetch(mfet_tables_t* t, const mfet_batch_shape_t* shape, const uint64_t* ids,
                        const int64_t* offsets, const int32_t* table_ids, mfet_stream_t stream);
 
+/* Gradient of the pooled output with respect to the rows of ONE slot's table (paper,
+ * Section 4.3: the pretrained tables are fine-tuned inside the ranking model, not frozen),
+ * as a sparse list: grad_rows = ascending distinct rows that the slot looked up,
+ * grad_vals[k, :] = sum over the lookups i of row grad_rows[k] of
+ *     c_i * grad_out[b(i), col_slot : col_slot + dim],
+ * c_i = 1 (SUM), 1/len(bag) (MEAN) or weights[i] (WSUM), accumulated in fp32 in input order.
+ *   shape, ids, offsets, weights, table_ids, pooling: as in the forward call
+ *   grad_out   dev f32[B, out_ld]: gradient of `out`
+ *   slot       which slot's table (0 <= slot < L); its table may live in HBM or host memory
+ *   grad_rows  dev i64[n], grad_vals dev f32[n, dim], n_rows dev i64[1]; n = number of IDs
+ *              of the slot's feature (at most the workspace capacity)
+ * Uses the workspace (the sort of the dedup). Errors: INVALID_ARG, WORKSPACE, CUDA. */
+MFET_API int mfet_embedding_bag_backward(mfet_tables_t* t, const mfet_batch_shape_t* shape, const uint64_t* ids,
+                                const int64_t* offsets, const float* weights, const int32_t* table_ids,
+                                const int32_t* pooling, const float* grad_out, int32_t slot,
+                                int64_t* grad_rows, float* grad_vals, int64_t* n_rows, mfet_stream_t stream);
+
 /* In-batch dedup of hashed rows, done before host reads so that each distinct
  * row crosses PCIe once (paper, Section 3.3 motivates keeping host traffic off
  * the latency path). uniq = ascending distinct values of rows[0..n);

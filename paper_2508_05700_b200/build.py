@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmfet.so")
-SOURCES = ["api.cu", "bag.cu", "hash_fill.cu", "dedup.cu", "hostpath.cu"]
+SOURCES = ["api.cu", "bag.cu", "hash_fill.cu", "dedup.cu", "hostpath.cu", "backward.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--fmad=true"]
 

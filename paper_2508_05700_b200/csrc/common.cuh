@@ -193,6 +193,7 @@ struct DedupArgs {
   int64_t* miss_rows;
   int64_t* n_miss;
   uint32_t* err;
+  const uint32_t** sorted_pos_out;  // optional: receives the array of original positions in sorted order
 };
 
 // Where the pooling kernel finds the rows of a host-table slot.
@@ -219,6 +220,11 @@ cudaError_t launch_bag_indirect(const BagParams& p, const IndirectParams& ip, cu
 // stage bit0: hash + dedup + probe + fetch into result set `set`; bit1: pool from it
 int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, int32_t feature, int32_t pooling,
                   uint32_t col, cudaStream_t side, int stage, int set);
+
+cudaError_t launch_backward(const uint32_t* sorted_pos, const int32_t* seg_start, const int64_t* n_unique, NSrc ns,
+                            const int64_t* offsets_f, int32_t batch, const float* weights, int32_t pooling,
+                            const float* grad_out, int64_t out_ld, uint32_t col, uint32_t dim, float* grad_vals,
+                            cudaStream_t s);
 
 // launch helpers implemented in the kernel files
 cudaError_t launch_hash(const uint64_t* ids, int64_t n, uint64_t seed, uint64_t rows, uint64_t magic,

@@ -328,6 +328,7 @@ __global__ void __launch_bounds__(kScanThreads) unique_write_kernel(NSrc ns, con
     if (i < n) {
       if (head[j]) {
         uniq[u] = (int64_t)k[j];
+        if (!PROBE && src) src[u] = (int32_t)i;  // where this row's run starts in the sorted order
         if (PROBE) {
           if (slot[j] < 0) {
             src[u] = -1 - (int32_t)m;
@@ -435,8 +436,9 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
     unique_count_kernel<false><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, none, nullptr, tile_counts, nblk2, tickets + 1,
                                                               a.n_unique, nullptr);
     unique_write_kernel<false><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, iin, nullptr, tile_counts, nblk2, a.uniq,
-                                                             a.inverse, nullptr, nullptr);
+                                                             a.inverse, a.src, nullptr);
   }
+  if (a.sorted_pos_out) *a.sorted_pos_out = iin;
   *launches += 2;
   return cudaGetLastError();
 }

@@ -35,7 +35,7 @@ EXPORTS = [
     "mfet_cache_build", "mfet_workspace_bytes", "mfet_set_workspace", "mfet_host_io_bytes",
     "mfet_embedding_bag_forward_host", "mfet_table_fill", "mfet_query_status", "mfet_set_option",
     "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static", "mfet_profile_read", "mfet_host_path_counts", "mfet_tables_set_version", "mfet_tables_version",
-    "mfet_host_prefetch",
+    "mfet_host_prefetch", "mfet_embedding_bag_backward",
 ]
 BATCH_IDS_ARE_ROWS, BATCH_PREFETCHED = 1, 2
 STATIC_DEDUP_MAX_IDS = 262144
@@ -85,6 +85,7 @@ _lib.mfet_host_path_counts.argtypes = [_P, C.POINTER(C.c_int64), C.POINTER(C.c_i
 _lib.mfet_tables_set_version.argtypes = [_P, C.c_uint64]
 _lib.mfet_tables_version.argtypes = [_P, C.POINTER(C.c_uint64)]
 _lib.mfet_host_prefetch.argtypes = [_P, C.POINTER(BatchShape), _P, _P, _P, _P]
+_lib.mfet_embedding_bag_backward.argtypes = [_P, C.POINTER(BatchShape), _P, _P, _P, _P, _P, _P, C.c_int32, _P, _P, _P, _P]
 _lib.mfet_launch_count.argtypes = [_P, C.POINTER(C.c_uint64)]
 for _n in EXPORTS:
     if _n not in ("mfet_row_bytes", "mfet_status_string"):
@@ -256,6 +257,14 @@ def mfet_host_prefetch(h, shape: BatchShape, ids, offsets, table_ids, stream=Non
     ti = _i32(table_ids)
     _check(_lib.mfet_host_prefetch(h, C.byref(shape), _ptr(ids), _ptr(offsets), ti.ctypes.data, _ptr(stream)),
            "mfet_host_prefetch")
+
+
+def mfet_embedding_bag_backward(h, shape: BatchShape, ids, offsets, weights, table_ids, pooling, grad_out, slot: int,
+                                grad_rows, grad_vals, n_rows, stream=None) -> None:
+    ti, po = _i32(table_ids), _i32(pooling)
+    _check(_lib.mfet_embedding_bag_backward(h, C.byref(shape), _ptr(ids), _ptr(offsets), _ptr(weights), ti.ctypes.data,
+                                            po.ctypes.data, _ptr(grad_out), slot, _ptr(grad_rows), _ptr(grad_vals),
+                                            _ptr(n_rows), _ptr(stream)), "mfet_embedding_bag_backward")
 
 
 def mfet_launch_count(h) -> int:
