@@ -1,0 +1,71 @@
+"""Parity at the full sizes of the five workloads, in the launch configuration that bench.py
+times (LookupEngine, full tables filled on the GPU, full batch): sampled output rows are
+recomputed one by one by the oracle from its procedural table values, the rest is checked
+through properties that hold at any size (finite, empty bags are zero, repeat runs identical)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2508_05700_b200 import inputs as gi
+from tests.helpers import assert_close, mfet
+
+pytestmark = pytest.mark.gpu
+
+
+def _host_rows_that_fit(w):
+    with open("/proc/meminfo") as fh:
+        avail = {l.split(":")[0]: int(l.split()[1]) * 1024 for l in fh}["MemAvailable"]
+    for t in w.tables:
+        if t.location == gi.LOC_HOST:
+            t.rows = min(t.rows, int(0.70 * avail) // (t.dim * 2))
+
+
+@pytest.mark.parametrize("config", [1, 2, 3, 4, 5])
+def test_full_size_sampled_parity(config):
+    m = mfet()
+    from paper_2508_05700_b200.runtime import LookupEngine
+    w = gi.make_workload(config)
+    _host_rows_that_fit(w)
+    need = sum(t.rows * m.row_bytes(t.dim, t.dtype) for t in w.tables if t.location == gi.LOC_DEVICE)
+    free, total = torch.cuda.mem_get_info()
+    if need > free - (6 << 30):
+        pytest.skip("not enough free device memory for workload %d" % config)
+    b = gi.make_batch(w, 0)
+    otabs = [orc.Table(rows=t.rows, dim=t.dim, dtype=t.dtype, hash_seed=t.hash_seed, value_key=t.value_key)
+             for t in w.tables]
+    with LookupEngine(w) as eng:
+        if eng.host_table_ids():
+            n_host = int(b.offsets[w.batch] - b.offsets[0])
+            eng.set_workspace(n_host + 4096)
+            eng.build_hot_cache(0, 0, int(w.tables[0].rows * w.cache_fraction))
+        d_ids = torch.from_numpy(b.ids.view(np.int64)).cuda()
+        d_off = torch.from_numpy(b.offsets).cuda()
+        d_w = None if b.weights is None else torch.from_numpy(b.weights).cuda()
+        out = torch.full((w.batch, w.out_dim), float("nan"), dtype=torch.float32, device="cuda")
+        eng.forward(d_ids, d_off, d_w, out)
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(eng.h) == 0
+        first = out.clone()
+        eng.forward(d_ids, d_off, d_w, out)
+        torch.cuda.synchronize()
+        assert torch.equal(first, out)                       # fixed summation order
+        assert bool(torch.isfinite(out).all())
+        # empty bags give exact zeros in their slot's columns (all samples, on the GPU)
+        lens = torch.from_numpy(np.diff(b.offsets).reshape(w.n_features, w.batch)).cuda()
+        col = 0
+        for s in range(w.n_slots):
+            D = w.tables[int(w.table_ids[s])].dim
+            empty = lens[int(w.slot_feature[s])] == 0
+            if bool(empty.any()):
+                assert not bool(out[empty, col:col + D].any())
+            col += D
+        # sampled rows against the oracle
+        rng = np.random.default_rng(100 + config)
+        pick = sorted(set(rng.integers(0, w.batch, 40).tolist()) | {0, w.batch - 1})
+        if config == 4:  # include the longest bag of the batch
+            pick = sorted(set(pick[:24]) | {int(np.diff(b.offsets).reshape(w.n_features, w.batch).max(axis=0).argmax())})
+        got = out[torch.tensor(pick, device="cuda")].cpu().numpy()
+    ref = orc.embedding_bag(otabs, w.batch, w.n_features, w.slot_feature, w.table_ids, w.pooling, b.ids, b.offsets,
+                            b.weights, samples=pick)
+    assert_close(got, ref, "workload %d at full size, %d sampled rows" % (config, len(pick)))
