@@ -38,8 +38,9 @@ void run(const uint8_t* table, const uint32_t* rows, int64_t n, uint32_t* out, i
   float ms; cudaEventElapsedTime(&ms, e0, e1); ms /= 10;
   printf("rowB=%d U=%d blocks/SM=%d threads=%d warps/SM=%d : %.1f us  %.0f GB/s\n", ROWB, U, blocks_per_sm, threads, blocks_per_sm * threads / 32, ms * 1e3, n * (double)ROWB / ms / 1e6);
 }
-int main() {
-  const uint64_t table_bytes = 40ull << 30;
+int main(int argc, char** argv) {
+  // table size in MiB (default 40 GiB: no L2 reuse; 64 MiB: every row read hits the 126 MB L2)
+  const uint64_t table_bytes = (argc > 1 ? (uint64_t)atoll(argv[1]) : 40960ull) << 20;
   const int64_t n = 16 << 20;  // rows gathered per launch (2 GiB at 128 B)
   uint8_t* table; uint32_t* rows; uint32_t* out;
   CK(cudaMalloc(&table, table_bytes)); CK(cudaMemset(table, 1, table_bytes));
