@@ -1,5 +1,6 @@
 // C-ABI boundary: argument checking, descriptor bookkeeping and launch
 // orchestration. No arithmetic of the lookup path happens on the host.
+#include <algorithm>
 #include <cstring>
 #include <new>
 
@@ -227,7 +228,8 @@ int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value) {
       t->prof_valid = false;
       return MFET_OK;
     case MFET_OPT_TILE:
-      if (value != 0 && value != 8 && value != 16 && value != 32 && value != 64) return MFET_ERR_INVALID_ARG;
+      if (value != 0 && value != 8 && value != 16 && value != 32 && value != 64 && value != 128)
+        return MFET_ERR_INVALID_ARG;
       t->tile = (int32_t)value;
       return MFET_OK;
     default: return MFET_ERR_INVALID_ARG;
@@ -375,7 +377,7 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
   p.group_policy = t->group_policy;
   // bags per block: full tiles once there is enough work to fill the GPU several times over
   const int64_t bags = (int64_t)B * L;
-  p.tile = bags >= 148LL * 8 * 64 ? 64 : (bags >= 148LL * 4 * 32 ? 32 : 16);
+  p.tile = bags >= 148LL * 16 * 128 ? 128 : (bags >= 16384 ? 64 : (bags >= 4096 ? 32 : 16));
   if (t->tile) p.tile = t->tile;
   p.tiles_per_slot = (B + p.tile - 1) / p.tile;
 
@@ -385,6 +387,10 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
   int n = 0;
   auto flush = [&]() -> int {
     if (n == 0) return MFET_OK;
+    // widest rows first: their blocks run longest, so they should not be the last to start
+    std::stable_sort(p.slot, p.slot + n, [](const SlotDev& a, const SlotDev& b) {
+      return (uint32_t)a.chunks * (a.dtype == MFET_INT4 ? 4u : 16u) > (uint32_t)b.chunks * (b.dtype == MFET_INT4 ? 4u : 16u);
+    });
     p.n_slots = n;
     if (launch_bag(p, stream) != cudaSuccess) return MFET_ERR_CUDA;
     t->launches += 1;

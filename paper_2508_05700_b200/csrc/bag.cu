@@ -217,7 +217,9 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
 
   // bags perm[q0 .. q1) of the tile, NG at a time
   auto open_bag = [&](int qb, BagCur& b) {
-    const int q = qb + grp;
+    // bags come in falling length: every other pass hands them out in reverse group order, so
+    // that no warp collects the longest bag of every pass
+    const int q = qb + ((((qb - q0) / NG) & 1) ? NG - 1 - grp : grp);
     b.have = q < q1;
     b.bi = b.have ? (int)perm[q] : 0;
     b.lo = 0;
@@ -410,7 +412,8 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   __shared__ int64_t soff[kMaxTile + 1];
   __shared__ int64_t sfeat[2];
   __shared__ uint8_t perm[kMaxTile];
-  __shared__ int scnt[2][16];
+  constexpr int kSortWarps = kMaxTile / 32;  // warps whose threads own one bag each in the ordering
+  __shared__ int scnt[kSortWarps][16];
   const int slot = blockIdx.x / p.tiles_per_slot;
   const int tile = blockIdx.x - slot * p.tiles_per_slot;
   const SlotDev& s = p.slot[slot];
@@ -419,7 +422,7 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   const long long* offs = reinterpret_cast<const long long*>(p.offsets) + (int64_t)s.feature * p.batch;
   if ((int)threadIdx.x <= nb) soff[threadIdx.x] = __ldcs(offs + b0 + threadIdx.x);
   if (IND && threadIdx.x < 2) sfeat[threadIdx.x] = offs[threadIdx.x ? p.batch : 0];
-  if (threadIdx.x >= 128 && threadIdx.x < 160) (&scnt[0][0])[threadIdx.x - 128] = 0;
+  if (threadIdx.x >= 128 && threadIdx.x < 128 + kSortWarps * 16) (&scnt[0][0])[threadIdx.x - 128] = 0;
   __syncthreads();
   int64_t feat_lo = 0;
   if constexpr (IND) {
@@ -440,7 +443,7 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   const int lane_ = threadIdx.x & 31, warp_ = threadIdx.x >> 5;
   bool have = false;
   int cls = 0, in_warp = 0;
-  if (warp_ < 2) {  // threads 0..63 own one bag each
+  if (warp_ < kSortWarps) {  // threads 0..kMaxTile-1 own one bag each
     have = (int)threadIdx.x < nb;
     if (have) {
       const int64_t l = soff[threadIdx.x + 1] - soff[threadIdx.x];
@@ -453,12 +456,17 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   }
   __syncthreads();
   if (have) {
-    int rank = in_warp + (warp_ ? scnt[0][cls] : 0);
-    for (int c2 = cls + 1; c2 < 16; ++c2) rank += scnt[0][c2] + scnt[1][c2];
+    int rank = in_warp;
+    for (int w2 = 0; w2 < warp_; ++w2) rank += scnt[w2][cls];
+    for (int c2 = cls + 1; c2 < 16; ++c2)
+#pragma unroll
+      for (int w2 = 0; w2 < kSortWarps; ++w2) rank += scnt[w2][c2];
     perm[rank] = (uint8_t)threadIdx.x;
   }
   __syncthreads();
-  int n_long = scnt[0][15] + scnt[1][15];
+  int n_long = 0;
+#pragma unroll
+  for (int w2 = 0; w2 < kSortWarps; ++w2) n_long += scnt[w2][15];
   if (p.group_policy == 1) n_long = 0;
   if (p.group_policy == 2) n_long = nb;
 
