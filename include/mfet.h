@@ -293,7 +293,7 @@ MFET_API int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits /*h
  * group per bag (best for short bags), 2 = one warp per bag (long bags). The
  * result is the same up to the order of fp32 additions. MFET_OPT_TILE: samples per
  * thread block of the pooling kernel: 0 = chosen from the batch size (default), or
- * 8 / 16 / 32 / 64. MFET_OPT_PROFILE: 1 = record CUDA events around the stages of
+ * 8 .. 128 (multiples of 32 suit the kernel best). MFET_OPT_PROFILE: 1 = record CUDA events around the stages of
  * the host-table path of every forward call (read them with mfet_profile_read). */
 MFET_API int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value);
 

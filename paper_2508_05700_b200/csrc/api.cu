@@ -228,8 +228,7 @@ int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value) {
       t->prof_valid = false;
       return MFET_OK;
     case MFET_OPT_TILE:
-      if (value != 0 && value != 8 && value != 16 && value != 32 && value != 64 && value != 128)
-        return MFET_ERR_INVALID_ARG;
+      if (value != 0 && (value < 8 || value > kMaxTile)) return MFET_ERR_INVALID_ARG;
       t->tile = (int32_t)value;
       return MFET_OK;
     default: return MFET_ERR_INVALID_ARG;

@@ -23,10 +23,8 @@
 #include "common.cuh"
 
 // Tunables (overridable at build time for sweeps): row loads kept in flight per
-// lane, the length from which a bag gets a whole warp, the minimum number of
-// resident blocks per SM (caps registers) and the accumulate flavour
-// (0 convert + scalar FMA, 1 packed f32x2 FMA, 2 mixed-precision add for
-// unweighted 16-bit tables).
+// lane, the length from which a bag gets a whole warp and the minimum number of
+// resident blocks per SM (caps registers).
 #ifndef MFET_BAG_U
 #define MFET_BAG_U 4
 #endif
@@ -35,9 +33,6 @@
 #endif
 #ifndef MFET_BAG_MINB
 #define MFET_BAG_MINB 5
-#endif
-#ifndef MFET_BAG_ACC
-#define MFET_BAG_ACC 1
 #endif
 
 namespace mfet {
@@ -75,7 +70,7 @@ __device__ __forceinline__ void fma2(unsigned long long& a, unsigned long long x
 // acc (E fp32 values as E/2 packed pairs) += w * (the 16-byte chunk v decoded to
 // fp32). The up-conversion of fp16 / bf16 is exact.
 template <int DT>
-__device__ __forceinline__ void accumulate(unsigned long long* acc, const uint4& v, float w, bool wsum) {
+__device__ __forceinline__ void accumulate(unsigned long long* acc, const uint4& v, float w) {
   if constexpr (DT == MFET_INT4) {
     // value = fma(code, scale, bias) in fp32 (one rounding), then acc += w * value
     const float2 sb = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
@@ -91,45 +86,9 @@ __device__ __forceinline__ void accumulate(unsigned long long* acc, const uint4&
       fma2(val, pack2(__float_as_uint(c0), __float_as_uint(c1)), s2);
       fma2(acc[j], val, w2);
     }
-    (void)wsum;
     return;
   }
   const uint32_t x[4] = {v.x, v.y, v.z, v.w};
-#if MFET_BAG_ACC == 0
-  float* a = reinterpret_cast<float*>(acc);
-  if constexpr (DT == MFET_F32) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) a[j] = fmaf(w, __uint_as_float(x[j]), a[j]);
-  } else if constexpr (DT == MFET_F16) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&x[j]));
-      a[2 * j] = fmaf(w, f.x, a[2 * j]);
-      a[2 * j + 1] = fmaf(w, f.y, a[2 * j + 1]);
-    }
-  } else {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      a[2 * j] = fmaf(w, bf16lo(x[j]), a[2 * j]);
-      a[2 * j + 1] = fmaf(w, bf16hi(x[j]), a[2 * j + 1]);
-    }
-  }
-#else
-#if MFET_BAG_ACC == 2
-  if (DT != MFET_F32 && !wsum) {  // acc += x with the 16-bit operand converted inside the add
-    float* a = reinterpret_cast<float*>(acc);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if constexpr (DT == MFET_F16)
-        asm("{.reg .b16 l, h; mov.b32 {l, h}, %2; add.rn.f32.f16 %0, l, %0; add.rn.f32.f16 %1, h, %1;}"
-            : "+f"(a[2 * j]), "+f"(a[2 * j + 1]) : "r"(x[j]));
-      else
-        asm("{.reg .b16 l, h; mov.b32 {l, h}, %2; add.rn.f32.bf16 %0, l, %0; add.rn.f32.bf16 %1, h, %1;}"
-            : "+f"(a[2 * j]), "+f"(a[2 * j + 1]) : "r"(x[j]));
-    }
-    return;
-  }
-#endif
   const unsigned long long w2 = pack2(__float_as_uint(w), __float_as_uint(w));
   if constexpr (DT == MFET_F32) {
     fma2(acc[0], pack2(x[0], x[1]), w2);
@@ -144,8 +103,6 @@ __device__ __forceinline__ void accumulate(unsigned long long* acc, const uint4&
 #pragma unroll
     for (int j = 0; j < 4; ++j) fma2(acc[j], pack2(x[j] << 16, x[j] & 0xFFFF0000u), w2);
   }
-#endif
-  (void)wsum;
 }
 
 // Combine the GG row groups of a bag group. While a lane holds more than one
@@ -329,7 +286,7 @@ __device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, 
         }
       }
 #pragma unroll
-      for (int k = 0; k < U; ++k) accumulate<DT>(acc, v[k], wk[k], wsum);
+      for (int k = 0; k < U; ++k) accumulate<DT>(acc, v[k], wk[k]);
     }
 
     // ---- end of the bag: combine row groups, scale, store ---------------------
