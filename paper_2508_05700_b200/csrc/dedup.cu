@@ -57,8 +57,18 @@ __device__ __forceinline__ bool last_block_arrives(uint32_t* ticket) {
 __device__ __forceinline__ void scan_digit_counts(uint32_t* hist, int nblk) {
   __shared__ uint32_t warp_tot[8];
   const int d = threadIdx.x;
+  // every load below is independent of the others: batches of 16 are issued together so that
+  // the pass costs nblk/16 memory round trips instead of nblk
   uint32_t tot = 0;
-  for (int b = 0; b < nblk; ++b) tot += __ldcg(hist + (size_t)b * 256 + d);
+  int b = 0;
+  for (; b + 16 <= nblk; b += 16) {
+    uint32_t v[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = __ldcg(hist + (size_t)(b + j) * 256 + d);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) tot += v[j];
+  }
+  for (; b < nblk; ++b) tot += __ldcg(hist + (size_t)b * 256 + d);
   const int lane = d & 31;
   uint32_t inc = tot;
 #pragma unroll
@@ -70,7 +80,18 @@ __device__ __forceinline__ void scan_digit_counts(uint32_t* hist, int nblk) {
   __syncthreads();
   uint32_t run = inc - tot;
   for (int w = 0; w < (d >> 5); ++w) run += warp_tot[w];
-  for (int b = 0; b < nblk; ++b) {
+  b = 0;
+  for (; b + 16 <= nblk; b += 16) {
+    uint32_t v[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = __ldcg(hist + (size_t)(b + j) * 256 + d);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      hist[(size_t)(b + j) * 256 + d] = run;
+      run += v[j];
+    }
+  }
+  for (; b < nblk; ++b) {
     const uint32_t v = __ldcg(hist + (size_t)b * 256 + d);
     hist[(size_t)b * 256 + d] = run;
     run += v;
@@ -131,55 +152,77 @@ __global__ void __launch_bounds__(kSortThreads) hist_kernel(NSrc ns, const uint6
   }
 }
 
-// Stable scatter of one tile by the current digit. Rounds of 256 keys keep the
-// input order: within a round, warps are ordered through per-warp digit counts
-// and lanes through match_any masks.
+// Stable scatter of one tile by the current digit. A thread holds one key of each of the
+// tile's rounds (round r = keys r*256 .. r*256+255 of the tile, so (round, warp, lane) is the
+// input order). Phase 1: per (round, warp) digit counts and every key's rank among the equal
+// digits of its warp, through match_any. Phase 2: thread d turns the 64 counts of digit d into
+// running offsets. Phase 3: position = tile's start for the digit + offset of (round, warp) +
+// rank. Two block barriers in all.
 __global__ void __launch_bounds__(kSortThreads) scatter_kernel(NSrc ns, const uint64_t* __restrict__ keys_in,
                                                                const uint32_t* __restrict__ idx_in,
                                                                uint64_t* __restrict__ keys_out,
                                                                uint32_t* __restrict__ idx_out, int shift,
                                                                const uint32_t* __restrict__ hist, int nblk) {
-  __shared__ uint32_t base[256];
-  __shared__ uint32_t wcnt[kSortThreads / 32][256];
+  constexpr int kWarps = kSortThreads / 32;
+  __shared__ uint16_t wcnt[kSortRounds][kWarps][256];  // counts, then offsets inside the tile (< 2048)
   int64_t lo;
   const int64_t n = resolve_n(ns, &lo);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  base[threadIdx.x] = hist[(size_t)blockIdx.x * 256 + threadIdx.x];
-#pragma unroll
-  for (int w = 0; w < kSortThreads / 32; ++w) wcnt[w][threadIdx.x] = 0;
-  __syncthreads();
   const int64_t tile0 = (int64_t)blockIdx.x * kSortTile;
   if (tile0 >= n) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t base = hist[(size_t)blockIdx.x * 256 + threadIdx.x];  // start of digit threadIdx.x for this tile
+  {
+    uint32_t* z = reinterpret_cast<uint32_t*>(&wcnt[0][0][0]);
+#pragma unroll
+    for (int j = 0; j < kSortRounds * kWarps * 256 / 2 / kSortThreads; ++j) z[j * kSortThreads + threadIdx.x] = 0u;
+  }
+  __syncthreads();
+  uint64_t k[kSortRounds];
+  uint32_t src[kSortRounds];
+  uint32_t dr[kSortRounds];  // digit | rank << 8 | valid << 16
+#pragma unroll
   for (int r = 0; r < kSortRounds; ++r) {
     const int64_t i = tile0 + r * kSortThreads + threadIdx.x;
     const bool valid = i < n;
-    uint64_t k = 0;
-    uint32_t src = 0;
+    k[r] = 0;
+    src[r] = 0;
     if (valid) {
-      k = keys_in[i];
-      src = idx_in ? idx_in[i] : (uint32_t)i;
+      k[r] = keys_in[i];
+      src[r] = idx_in ? idx_in[i] : (uint32_t)i;
     }
-    const uint32_t d = (uint32_t)(k >> shift) & 255u;
-    const uint32_t tag = valid ? d : (256u + (uint32_t)lane);  // invalid lanes match nobody
-    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, tag);
-    const uint32_t rank = __popc(peers & ((1u << lane) - 1u));
-    if (valid && rank == 0) wcnt[warp][d] = __popc(peers);
-    __syncthreads();
-    if (valid) {
-      uint32_t pos = base[d] + rank;
-      for (int w = 0; w < warp; ++w) pos += wcnt[w][d];
-      keys_out[pos] = k;
-      idx_out[pos] = src;
-    }
-    __syncthreads();
-    uint32_t add = 0;
+  }
 #pragma unroll
-    for (int w = 0; w < kSortThreads / 32; ++w) {
-      add += wcnt[w][threadIdx.x];
-      wcnt[w][threadIdx.x] = 0;
+  for (int r = 0; r < kSortRounds; ++r) {
+    const bool valid = tile0 + r * kSortThreads + threadIdx.x < n;
+    const uint32_t d = (uint32_t)(k[r] >> shift) & 255u;
+    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, valid ? d : (256u + (uint32_t)lane));  // invalid lanes match nobody
+    const uint32_t rank = __popc(peers & ((1u << lane) - 1u));
+    if (valid && rank == 0) wcnt[r][warp][d] = (uint16_t)__popc(peers);
+    dr[r] = d | (rank << 8) | (valid ? 1u << 16 : 0u);
+  }
+  __syncthreads();
+  {
+    uint32_t run = 0;  // thread d: exclusive running sum of digit d over (round, warp)
+#pragma unroll
+    for (int r = 0; r < kSortRounds; ++r)
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        const uint32_t c = wcnt[r][w][threadIdx.x];
+        wcnt[r][w][threadIdx.x] = (uint16_t)run;
+        run += c;
+      }
+  }
+  __shared__ uint32_t sbase[256];
+  sbase[threadIdx.x] = base;
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < kSortRounds; ++r) {
+    if (dr[r] >> 16) {
+      const uint32_t d = dr[r] & 255u;
+      const uint32_t pos = sbase[d] + wcnt[r][warp][d] + ((dr[r] >> 8) & 255u);
+      keys_out[pos] = k[r];
+      idx_out[pos] = src[r];
     }
-    base[threadIdx.x] += add;
-    __syncthreads();
   }
 }
 
