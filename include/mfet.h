@@ -265,6 +265,18 @@ MFET_API int mfet_embedding_bag_forward_host(mfet_tables_t* t, const mfet_batch_
                                     const int32_t* pooling, float* out_host, void* dev_io,
                                     uint64_t dev_io_bytes, mfet_stream_t stream);
 
+/* The same without the final wait: the copies and kernels are queued on `stream` and the call
+ * returns. `out_host` is complete once `stream` has been synchronised (or an event recorded
+ * after the call has fired); the host buffers must be pinned and must stay untouched until
+ * then, and `dev_io` must not be shared with another call in flight. Two calls on two
+ * streams with two `dev_io` buffers overlap one step's result copy with the next step's
+ * input copy and kernels. */
+MFET_API int mfet_embedding_bag_forward_host_async(mfet_tables_t* t, const mfet_batch_shape_t* shape,
+                                    const uint64_t* ids_host, const int64_t* offsets_host,
+                                    const float* weights_host, int64_t nnz, const int32_t* table_ids,
+                                    const int32_t* pooling, float* out_host, void* dev_io,
+                                    uint64_t dev_io_bytes, mfet_stream_t stream);
+
 /* Synthetic table contents (the paper's tables are pretrained weights that are
  * not public; this counter-based generator stands in for them):
  *   k = r*dim + d;  u = splitmix64(value_key + k)

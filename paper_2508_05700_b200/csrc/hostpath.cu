@@ -298,10 +298,10 @@ int mfet_host_io_bytes(const mfet_tables_t* t, const mfet_batch_shape_t* shape, 
   return MFET_OK;
 }
 
-int mfet_embedding_bag_forward_host(mfet_tables_t* t, const mfet_batch_shape_t* shape, const uint64_t* ids_host,
-                                    const int64_t* offsets_host, const float* weights_host, int64_t nnz,
-                                    const int32_t* table_ids, const int32_t* pooling, float* out_host, void* dev_io,
-                                    uint64_t dev_io_bytes, mfet_stream_t stream_) {
+static int forward_host_impl(mfet_tables_t* t, const mfet_batch_shape_t* shape, const uint64_t* ids_host,
+                             const int64_t* offsets_host, const float* weights_host, int64_t nnz,
+                             const int32_t* table_ids, const int32_t* pooling, float* out_host, void* dev_io,
+                             uint64_t dev_io_bytes, mfet_stream_t stream_, bool wait) {
   uint64_t need = 0;
   int rc = mfet_host_io_bytes(t, shape, table_ids, nnz, &need);
   if (rc != MFET_OK) return rc;
@@ -333,12 +333,28 @@ int mfet_embedding_bag_forward_host(mfet_tables_t* t, const mfet_batch_shape_t* 
     if (rc == MFET_OK) {
       ok = cudaMemcpyAsync(out_host, d_out, (size_t)shape->batch * out_ld * 4, cudaMemcpyDeviceToHost, stream) ==
            cudaSuccess;
-      ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+      if (wait) ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
     }
   }
   if (prev != t->device) cudaSetDevice(prev);
   if (rc != MFET_OK) return rc;
   return ok ? MFET_OK : MFET_ERR_CUDA;
+}
+
+int mfet_embedding_bag_forward_host(mfet_tables_t* t, const mfet_batch_shape_t* shape, const uint64_t* ids_host,
+                                    const int64_t* offsets_host, const float* weights_host, int64_t nnz,
+                                    const int32_t* table_ids, const int32_t* pooling, float* out_host, void* dev_io,
+                                    uint64_t dev_io_bytes, mfet_stream_t stream) {
+  return forward_host_impl(t, shape, ids_host, offsets_host, weights_host, nnz, table_ids, pooling, out_host, dev_io,
+                           dev_io_bytes, stream, true);
+}
+
+int mfet_embedding_bag_forward_host_async(mfet_tables_t* t, const mfet_batch_shape_t* shape, const uint64_t* ids_host,
+                                          const int64_t* offsets_host, const float* weights_host, int64_t nnz,
+                                          const int32_t* table_ids, const int32_t* pooling, float* out_host,
+                                          void* dev_io, uint64_t dev_io_bytes, mfet_stream_t stream) {
+  return forward_host_impl(t, shape, ids_host, offsets_host, weights_host, nnz, table_ids, pooling, out_host, dev_io,
+                           dev_io_bytes, stream, false);
 }
 
 }  // extern "C"

@@ -35,7 +35,7 @@ EXPORTS = [
     "mfet_cache_build", "mfet_workspace_bytes", "mfet_set_workspace", "mfet_host_io_bytes",
     "mfet_embedding_bag_forward_host", "mfet_table_fill", "mfet_query_status", "mfet_set_option",
     "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static", "mfet_profile_read", "mfet_host_path_counts", "mfet_tables_set_version", "mfet_tables_version",
-    "mfet_host_prefetch", "mfet_embedding_bag_backward",
+    "mfet_host_prefetch", "mfet_embedding_bag_backward", "mfet_embedding_bag_forward_host_async",
 ]
 BATCH_IDS_ARE_ROWS, BATCH_PREFETCHED = 1, 2
 STATIC_DEDUP_MAX_IDS = 262144
@@ -76,6 +76,7 @@ _lib.mfet_set_workspace.argtypes = [_P, _P, C.c_uint64, C.c_int64]
 _lib.mfet_host_io_bytes.argtypes = [_P, C.POINTER(BatchShape), _P, C.c_int64, C.POINTER(C.c_uint64)]
 _lib.mfet_embedding_bag_forward_host.argtypes = [_P, C.POINTER(BatchShape), _P, _P, _P, C.c_int64, _P, _P, _P,
                                                  _P, C.c_uint64, _P]
+_lib.mfet_embedding_bag_forward_host_async.argtypes = _lib.mfet_embedding_bag_forward_host.argtypes
 _lib.mfet_table_fill.argtypes = [_P, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
                                  C.c_uint32, _P]
 _lib.mfet_query_status.argtypes = [_P, C.POINTER(C.c_uint32), C.c_int32]
@@ -211,6 +212,15 @@ def mfet_embedding_bag_forward_host(h, shape: BatchShape, ids_host, offsets_host
                                                 _ptr(weights_host), nnz, ti.ctypes.data, po.ctypes.data,
                                                 _ptr(out_host), _ptr(dev_io), dev_io_bytes, _ptr(stream)),
            "mfet_embedding_bag_forward_host")
+
+
+def mfet_embedding_bag_forward_host_async(h, shape: BatchShape, ids_host, offsets_host, weights_host, nnz: int,
+                                          table_ids, pooling, out_host, dev_io, dev_io_bytes: int, stream=None) -> None:
+    ti, po = _i32(table_ids), _i32(pooling)
+    _check(_lib.mfet_embedding_bag_forward_host_async(h, C.byref(shape), _ptr(ids_host), _ptr(offsets_host),
+                                                      _ptr(weights_host), nnz, ti.ctypes.data, po.ctypes.data,
+                                                      _ptr(out_host), _ptr(dev_io), dev_io_bytes, _ptr(stream)),
+           "mfet_embedding_bag_forward_host_async")
 
 
 def mfet_table_fill(data, row0: int, n_rows: int, dim: int, dtype: int, row_stride_bytes: int, value_key: int,
