@@ -298,6 +298,9 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
     from paper_2508_05700_b200.runtime import LookupEngine
 
     w = gi.make_workload(config, rows_scale=args.rows_scale)
+    if args.alpha is not None:  # e.g. 0 = uniform IDs: no row repeats, the pure random-gather case
+        w.alpha = np.full(w.n_features, float(args.alpha))
+        w.name += ", Zipf alpha overridden to %g" % args.alpha
     scaled_host = False
     fits = host_rows_that_fit(w)
     if fits:
@@ -533,6 +536,7 @@ def main():
     ap.add_argument("--no-hybrid", action="store_true", help="skip the hybrid workload after the default one")
     ap.add_argument("--impl", default="mfet", choices=["mfet", "reference"])
     ap.add_argument("--rows-scale", type=float, default=1.0, help="shrink table rows (reported in config)")
+    ap.add_argument("--alpha", type=float, default=None, help="override the Zipf exponent of every feature (0 = uniform IDs)")
     ap.add_argument("--batches", type=int, default=8, help="distinct batches rotated through")
     ap.add_argument("--load-seconds", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")

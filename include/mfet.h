@@ -149,8 +149,11 @@ MFET_API int mfet_hash_ids(const mfet_tables_t* t, int32_t table_id, const uint6
  *   out      dev f32[B, out_ld]; the columns of all slots are fully overwritten
  * Slots whose table is in host memory run on the library's internal stream
  * (dedup -> cache probe -> host fetch -> pool), overlapped with the others and
- * joined back into `stream`; they need a workspace (mfet_set_workspace) and
- * `nnz_hint`-free operation: sizes are taken from the workspace capacity.
+ * joined back into `stream`; they need a workspace (mfet_set_workspace). The
+ * host never learns how many IDs such a slot has: the kernels read the count from
+ * `offsets` and are sized by the workspace capacity; a slot with more IDs than
+ * that sets MFET_DEV_CAPACITY and its columns are written as zeros.
+ * Calls on one handle must not overlap on the GPU when they use the workspace.
  * Errors: INVALID_ARG, NOT_REGISTERED, WORKSPACE, CUDA. */
 MFET_API int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape,
                                const uint64_t* ids, const int64_t* offsets, const float* weights,
