@@ -314,6 +314,10 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
 
     dev = torch.cuda.current_device()
     eng = LookupEngine(w, device=dev)
+    if args.tile:
+        m.mfet_set_option(eng.h, m.OPT_TILE, args.tile)
+    if args.stage_ids:
+        m.mfet_set_option(eng.h, m.OPT_STAGE_IDS, args.stage_ids)
     stream = torch.cuda.current_stream()
     host_tabs = eng.host_table_ids()
     cached_rows = 0
@@ -540,6 +544,8 @@ def main():
     ap.add_argument("--batches", type=int, default=8, help="distinct batches rotated through")
     ap.add_argument("--load-seconds", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tile", type=int, default=0, help="samples per block of the pooling kernel (0 = library default)")
+    ap.add_argument("--stage-ids", type=int, default=0, help="IDs staged per pass of the pooling kernel (0 = library default)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -48,7 +48,7 @@ enum { MFET_POOL_SUM = 0, MFET_POOL_MEAN = 1, MFET_POOL_WSUM = 2 };
 enum { MFET_LOC_DEVICE = 0, MFET_LOC_HOST = 1 };
 enum { MFET_VAL_NORMAL = 0, MFET_VAL_GRID = 1 };
 enum { MFET_BATCH_IDS_ARE_ROWS = 1, MFET_BATCH_PREFETCHED = 2 }; /* mfet_batch_shape_t.flags */
-enum { MFET_OPT_GROUP_POLICY = 1, MFET_OPT_TILE = 2, MFET_OPT_PROFILE = 3 };
+enum { MFET_OPT_GROUP_POLICY = 1, MFET_OPT_TILE = 2, MFET_OPT_PROFILE = 3, MFET_OPT_STAGE_IDS = 4 };
 
 enum {
   MFET_OK = 0,
@@ -308,7 +308,11 @@ MFET_API int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits /*h
  * group per bag (best for short bags), 2 = one warp per bag (long bags). The
  * result is the same up to the order of fp32 additions. MFET_OPT_TILE: samples per
  * thread block of the pooling kernel: 0 = chosen from the batch size (default), or
- * 8 .. 128 (multiples of 32 suit the kernel best). MFET_OPT_PROFILE: 1 = record CUDA events around the stages of
+ * 8 .. 128 (multiples of 32 suit the kernel best). MFET_OPT_STAGE_IDS: how many IDs of a
+ * tile the pooling kernel hashes into shared memory at a time: 0 = default, or
+ * 32 .. 8192; a tile with more IDs is pooled in several passes and a bag cut by a pass
+ * boundary continues from its partial sum (same result up to the order of fp32
+ * additions). MFET_OPT_PROFILE: 1 = record CUDA events around the stages of
  * the host-table path of every forward call (read them with mfet_profile_read). */
 MFET_API int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value);
 

@@ -231,6 +231,10 @@ int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value) {
       if (value != 0 && (value < 8 || value > kMaxTile)) return MFET_ERR_INVALID_ARG;
       t->tile = (int32_t)value;
       return MFET_OK;
+    case MFET_OPT_STAGE_IDS:
+      if (value != 0 && (value < 32 || value > kStageMax)) return MFET_ERR_INVALID_ARG;
+      t->stage_cap = (int32_t)value;
+      return MFET_OK;
     default: return MFET_ERR_INVALID_ARG;
   }
 }
@@ -378,6 +382,7 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
   const int64_t bags = (int64_t)B * L;
   p.tile = bags >= 148LL * 16 * 128 ? 128 : (bags >= 16384 ? 64 : (bags >= 4096 ? 32 : 16));
   if (t->tile) p.tile = t->tile;
+  p.stage_cap = t->stage_cap;
   p.tiles_per_slot = (B + p.tile - 1) / p.tile;
 
   // host-table slots go to the side stream, forked from and joined to `stream`
@@ -436,7 +441,7 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
         uint8_t lg = 1;
         while ((1u << lg) < ch) ++lg;
         sd.lpr_log2 = lg;
-        sd.narrow = (tb.desc.rows * (tb.stride >> 4)) <= 0xFFFFFFFFULL ? 1 : 0;
+        sd.narrow = (tb.desc.rows <= 0xFFFFFFFFULL && tb.stride <= 0xFFFFFFFFULL) ? 1 : 0;
       }
     }
     col += tb.desc.dim;

@@ -1,38 +1,46 @@
 // K-bag: fused hash -> gather -> pool -> concatenated store, all device-table
 // slots of a batch in one launch.
 //
-// Work split. A block takes one (slot, tile of up to 64 consecutive samples);
-// the tile's CSR offsets are staged in shared memory and its bags are ordered by
-// falling length class. Inside the block a BAG GROUP of GL lanes owns one bag at
-// a time. A table row is 16-byte chunks; LPR lanes (a ROW GROUP) read one row
-// with one 16-byte load each, so a bag group reads GL/LPR rows per load
-// instruction. Long bags get GL = 32 (the whole warp streams one bag), all other
-// bags GL = LPR (several bags per warp, no cross-lane reduction at all); thanks
-// to the ordering the bag groups of a warp work on bags of similar length.
+// Work split. A block takes one (slot, tile of up to 128 consecutive samples).
+// The IDs of a tile are one contiguous range of the CSR arrays, so the block
+// first STAGES them: all 256 threads stream the range with coalesced loads, hash
+// every ID to its table row and park the 32-bit row index (and the weight) in
+// shared memory. The hashing of the whole tile therefore runs with full memory
+// parallelism and before any row is requested; the gather that follows has no
+// load that depends on another global load, and its inner loop is little more
+// than shared-memory read, address, 16-byte load and the fp32 adds.
 //
-// The work of a bag group is a sequence of ROUNDS of GL IDs. In a round every
-// lane hashes one ID (coalesced 8-byte loads, prefetched one round ahead so the
-// ID latency hides behind the previous round's rows), the row offsets travel by
-// shuffle to the row group that loads them, U loads are in flight per lane, and
-// batches of loads whose rows exist in every bag group of the warp run without
-// predicates. Accumulation is fp32 (packed two-wide FMA); row groups are
-// combined by a shuffle reduce-scatter so that every lane ends with a distinct
-// piece of the output row and the store is one coalesced segment. The order of
-// additions depends only on the inputs and the tile configuration, never on
+// Gather. A table row is 16-byte chunks; LPR lanes (a ROW GROUP) read one row
+// with one 16-byte load each. The tile's bags are ordered: long bags first, then
+// the others by falling length (counting sort). A long bag gets a whole warp
+// (its 32/LPR row groups stride over the bag's rows and are combined by a
+// shuffle reduce-scatter, so that every lane ends with a distinct piece of the
+// output row); every other bag is owned by one row group (32/LPR bags of nearly
+// equal length per warp, no cross-lane reduction at all). Warps take their next
+// bags from a shared counter. The steps that all lanes of a warp have in common
+// run without predicates in batches of U loads per lane; accumulation is fp32
+// (packed two-wide FMA).
+//
+// A tile whose IDs do not fit the staging buffer is processed in WINDOWS of the
+// buffer's capacity; a bag cut by a window boundary continues from the partial
+// sum that its earlier piece left in the output row. The order of additions
+// depends only on the inputs, the tile size and the staging capacity, never on
 // timing.
+#include <atomic>
+
 #include "common.cuh"
 
 // Tunables (overridable at build time for sweeps): row loads kept in flight per
 // lane, the length from which a bag gets a whole warp and the minimum number of
 // resident blocks per SM (caps registers).
 #ifndef MFET_BAG_U
-#define MFET_BAG_U 4
+#define MFET_BAG_U 8
 #endif
 #ifndef MFET_BAG_LONG
-#define MFET_BAG_LONG 64
+#define MFET_BAG_LONG 32
 #endif
 #ifndef MFET_BAG_MINB
-#define MFET_BAG_MINB 5
+#define MFET_BAG_MINB 4
 #endif
 
 namespace mfet {
@@ -41,6 +49,7 @@ namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kLongBag = MFET_BAG_LONG;  // bags at least this long get a whole warp
+static_assert(kLongBag >= 1 && kLongBag <= 32, "the ordering has one lane per shorter length");
 
 // A lane's piece of a row: 16 bytes (4 fp32 or 8 fp16/bf16 values), or for INT4 rows
 // 4 bytes (8 four-bit codes) plus the row's fp16 scale/bias pair.
@@ -133,253 +142,324 @@ struct ReduceScatter {
   }
 };
 
-// One bag of a bag group, as the round loop sees it.
-struct BagCur {
-  int64_t lo;   // first ID of the bag
-  int len;      // its length (0 when this group has no bag)
-  int bi;       // index inside the tile
-  int maxlen;   // longest / shortest bag among the warp's bag groups: the warp
-  int minlen;   // runs maxlen rows, the first minlen of them without predicates
-  bool have;
+
+// What a warp needs to know about the block's staging window. The window's bags
+// are listed long ones first, then by falling length: entry q has the window
+// position of the bag's first staged row, the number of its rows in the window
+// and the bag's index in the tile (plus kNotFirst when an earlier window held the
+// start of the bag and kNotLast when a later one holds its end).
+constexpr int kNotFirst = 0x100, kNotLast = 0x200;
+struct Win {
+  const uint32_t* srow;   // staged row index (IND: dedup source index) per window position
+  const uint32_t* shi;    // its upper half, for tables of more than 2^32-1 rows
+  const float* sw;        // staged weight per window position (weighted slots)
+  const int* spos;        // per listed bag, see above
+  const int* slen;
+  const int* sbag;
+  int* next;              // shared work counter
+  const int64_t* soff;    // the tile's CSR offsets
+  int nbw;                // bags listed
+  int n_long;             // the first n_long of them get a whole warp
+  int b0;                 // first sample of the tile
 };
 
-// IND = false: rows come from the slot's table by hashing the ID.
-// IND = true : rows of a host-table slot come from the HBM cache or the staging
-//              buffer, through the dedup inverse map (feat_lo = first ID of the
-//              slot's feature, so that positions are slot-local).
-template <int DT, int LPR, int GL, bool IND>
-__device__ __forceinline__ void pool_tile(const BagParams& p, const SlotDev& s, const int64_t* soff,
-                                          int b0, const uint8_t* perm, int q0, int q1,
-                                          const IndirectParams& ip, int64_t feat_lo) {
-  constexpr int E = ChunkElems<DT>::value;
-  constexpr int GG = GL / LPR;          // row groups per bag group
-  constexpr int NG = 256 / GL;          // bag groups per block
-  constexpr int U = LPR < MFET_BAG_U ? LPR : MFET_BAG_U;  // row loads in flight per lane
-  constexpr int NF = (E / GG) > 0 ? (E / GG) : 1;         // values a lane stores
-
-  const int lane = threadIdx.x & 31;
-  const int gl = lane & (GL - 1);
-  const int sub = gl / LPR;
-  const int c = gl & (LPR - 1);
-  const int grp = threadIdx.x / GL;
-  const bool all_chunks = (int)s.chunks == LPR;  // no idle chunk lanes
-  const bool chunk_ok = c < (int)s.chunks;
-  const bool wsum = s.pooling == MFET_POOL_WSUM;
-  const bool pre = (p.flags & 1u) != 0;
-  const bool narrow = !IND && s.narrow != 0;
-  const uint8_t* tbase = s.table + c * ChunkElems<DT>::bytes;  // IND: s.table = byte offset of the column block
-  const uint8_t* mbase = s.table + s.meta_off;               // INT4: the row's scale/bias pair
-  const uint64_t stride16 = s.stride >> 4;
-  const unsigned long long* ids = reinterpret_cast<const unsigned long long*>(p.ids);
-
-  // bags perm[q0 .. q1) of the tile, NG at a time
-  auto open_bag = [&](int qb, BagCur& b) {
-    // bags come in falling length: every other pass hands them out in reverse group order, so
-    // that no warp collects the longest bag of every pass
-    const int q = qb + ((((qb - q0) / NG) & 1) ? NG - 1 - grp : grp);
-    b.have = q < q1;
-    b.bi = b.have ? (int)perm[q] : 0;
-    b.lo = 0;
-    b.len = 0;
-    if (b.have) {
-      b.lo = soff[b.bi];
-      int64_t l = soff[b.bi + 1] - b.lo;
-      if (l < 0) {
-        if (gl == 0) atomicOr(p.err, (uint32_t)MFET_DEV_OFFSETS);
-        l = 0;
-      }
-      b.len = l > 0x7FFFFFFF ? 0x7FFFFFFF : (int)l;
+// Where this lane's chunk (and, INT4, the scale/bias pair) of a staged row is.
+// Direct tables: base + row * stride. IND: the dedup source index selects the
+// cache (>= 0) or the staging buffer of fetched rows (< 0: -1 - index).
+template <bool IND>
+struct RowAddr {
+  const uint8_t* tbase;   // table (IND: cache rows) + this lane's chunk offset
+  const uint8_t* mbase;   // same + the offset of the scale/bias pair
+  const uint8_t* tbase2;  // IND: the fetched-rows variants
+  const uint8_t* mbase2;
+  uint64_t stride;
+  uint32_t stride32;
+  bool wide;              // row index or stride beyond 32 bits
+  // the common case: row index and stride fit 32 bits
+  __device__ __forceinline__ void get_narrow(uint32_t lo, const uint8_t*& chunk, const uint8_t*& meta) const {
+    if constexpr (IND) {
+      get(lo, 0u, chunk, meta);
+    } else {
+      const uint64_t off = (uint64_t)lo * stride32;
+      chunk = tbase + off;
+      meta = mbase + off;
     }
-    b.maxlen = __reduce_max_sync(kFull, b.len);
-    b.minlen = __reduce_min_sync(kFull, b.len);
-  };
-  // the ID (or, IND, the row location) and weight of position base+gl of a bag
-  auto fetch = [&](const BagCur& b, int base, uint64_t& id, float& w) {
-    id = 0;
-    w = 1.f;
-    if (base + gl < b.len) {
-      const int64_t i = b.lo + base + gl;
-      if constexpr (IND) id = (uint32_t)__ldg(ip.inverse + (i - feat_lo));
-      else id = __ldcs(ids + i);
-      if (wsum) w = __ldcs(p.weights + i);
+  }
+  __device__ __forceinline__ void get(uint32_t lo, uint32_t hi, const uint8_t*& chunk, const uint8_t*& meta) const {
+    if constexpr (IND) {
+      const bool cached = (int32_t)lo >= 0;
+      const uint64_t off = (uint64_t)(cached ? lo : ~lo) * stride32;
+      chunk = (cached ? tbase : tbase2) + off;
+      meta = (cached ? mbase : mbase2) + off;
+    } else {
+      const uint64_t off = wide ? (((uint64_t)hi << 32) | lo) * stride : (uint64_t)lo * stride32;
+      chunk = tbase + off;
+      meta = mbase + off;
     }
-  };
+  }
+};
 
-  if (q0 >= q1) return;
-  BagCur cur;
-  open_bag(q0, cur);
-  int qb = q0, base = 0;
-  uint64_t id_c;
-  float w_c;
-  fetch(cur, 0, id_c, w_c);
-
-  unsigned long long acc[E / 2];
+// N consecutive steps of a lane: N row chunks are requested, then added to acc.
+// srow/shi/sw point at the lane's first of these steps; a step is GG staged
+// entries further than the one before. WS: the slot is weighted (a compile-time
+// copy of the flag for the common path). PRED = false: every lane has all N
+// steps, the table is narrow and every staged row is a row. PRED = true: the
+// lane has only `left` of the N steps (possibly none or all of them), and a
+// staged row may be the "no row" sentinel or lie outside this lane's chunks;
+// what is not loaded counts as zeros.
+template <int DT, int GG, bool IND, int N, bool PRED, bool WS>
+__device__ __forceinline__ void run_steps(const uint32_t* srow, const uint32_t* shi, const float* sw,
+                                          const RowAddr<IND>& ra, bool wsum, int left, bool chunk_ok,
+                                          unsigned long long* acc) {
+  uint4 v[N];
 #pragma unroll
-  for (int j = 0; j < E / 2; ++j) acc[j] = 0ull;
-
-  while (true) {
-    // ---- what comes after this round; its IDs are requested now -------------
-    const bool last_round = base + GL >= cur.maxlen;  // warp-uniform
-    BagCur nxt = cur;
-    int nbase = base + GL, nqb = qb;
-    bool more = true;
-    if (last_round) {
-      nqb = qb + NG;
-      nbase = 0;
-      more = nqb < q1;
-      if (more) open_bag(nqb, nxt);
-    }
-    uint64_t id_n = 0;
-    float w_n = 1.f;
-    if (more) fetch(nxt, nbase, id_n, w_n);
-
-    // ---- this round: every lane of the bag group resolves one row ------------
-    uint64_t off16 = ~0ULL;  // sentinel: no row
-    if (base + gl < cur.len) {
-      if constexpr (IND) {
-        const int32_t sidx = __ldg(ip.src + (uint32_t)id_c);
-        const uint8_t* rowp = sidx >= 0 ? ip.cache_data + (uint64_t)sidx * ip.row_bytes
-                                        : ip.staging + (uint64_t)(-1 - sidx) * ip.row_bytes;
-        off16 = reinterpret_cast<uint64_t>(rowp) >> 4;
-      } else {
-        const uint64_t row = pre ? id_c : mod_rows(splitmix64(id_c ^ s.seed), s.rows, s.magic);
-        if (row < s.rows) off16 = row * stride16;
-        else atomicOr(p.err, (uint32_t)MFET_DEV_ROW_RANGE);
-      }
-    }
-    const uint32_t off_lo = (uint32_t)off16, off_hi = (uint32_t)(off16 >> 32);
-    const int cnt = min(GL, cur.maxlen - base);                 // IDs of the longest group
-    const int full = all_chunks ? min(GL, cur.minlen - base) : 0;  // IDs that every group has
-#pragma unroll
-    for (int u0 = 0; u0 < LPR; u0 += U) {
-      if (u0 * GG >= cnt) break;
-      uint4 v[U];
-      float wk[U];
-      if ((u0 + U) * GG <= full && !pre) {
-        // every lane has a row in each of the U steps: no predicates
-#pragma unroll
-        for (int k = 0; k < U; ++k) {
-          const int src = (u0 + k) * GG + sub;
-          const uint32_t o_lo = __shfl_sync(kFull, off_lo, src, GL);
-          const uint32_t o_hi = narrow ? 0u : __shfl_sync(kFull, off_hi, src, GL);
-          wk[k] = wsum ? __shfl_sync(kFull, w_c, src, GL) : 1.f;
-          const uint64_t ro = (((uint64_t)o_hi << 32) | o_lo) << 4;
-          v[k] = load_chunk<DT>(tbase + ro, mbase + ro);
-        }
-      } else {
-#pragma unroll
-        for (int k = 0; k < U; ++k) {
-          const int src = (u0 + k) * GG + sub;
-          const uint32_t o_lo = __shfl_sync(kFull, off_lo, src, GL);
-          uint32_t o_hi = 0;
-          bool valid;
-          if (narrow) {
-            valid = o_lo != 0xFFFFFFFFu;
-          } else {
-            o_hi = __shfl_sync(kFull, off_hi, src, GL);
-            valid = (o_lo & o_hi) != 0xFFFFFFFFu;
-          }
-          wk[k] = wsum ? __shfl_sync(kFull, w_c, src, GL) : 1.f;
-          v[k] = make_uint4(0u, 0u, 0u, 0u);
-          const uint64_t ro = (((uint64_t)o_hi << 32) | o_lo) << 4;
-          if (valid && chunk_ok) v[k] = load_chunk<DT>(tbase + ro, mbase + ro);
+  for (int j = 0; j < N; ++j) {
+    const uint8_t *a, *m;
+    if constexpr (PRED) {
+      v[j] = make_uint4(0u, 0u, 0u, 0u);
+      if (j < left && chunk_ok) {
+        const uint32_t lo = srow[j * GG];
+        const uint32_t hi = (!IND && ra.wide) ? shi[j * GG] : 0u;
+        if (IND || (ra.wide ? (lo & hi) != 0xFFFFFFFFu : lo != 0xFFFFFFFFu)) {
+          ra.get(lo, hi, a, m);
+          v[j] = load_chunk<DT>(a, m);
         }
       }
-#pragma unroll
-      for (int k = 0; k < U; ++k) accumulate<DT>(acc, v[k], wk[k]);
+    } else {
+      ra.get_narrow(srow[j * GG], a, m);
+      v[j] = load_chunk<DT>(a, m);
     }
-
-    // ---- end of the bag: combine row groups, scale, store ---------------------
-    if (last_round) {
-      float a[E];
+  }
 #pragma unroll
-      for (int j = 0; j < E / 2; ++j) {
-        a[2 * j] = __uint_as_float((uint32_t)acc[j]);
-        a[2 * j + 1] = __uint_as_float((uint32_t)(acc[j] >> 32));
-        acc[j] = 0ull;
-      }
-      int off = 0;
-      bool writer = cur.have && chunk_ok;
-      ReduceScatter<E, 0, GG, LPR>::run(a, sub, off, writer);
-      if (s.pooling == MFET_POOL_MEAN && cur.len > 0) {
-        const float fl = (float)cur.len;
-#pragma unroll
-        for (int j = 0; j < NF; ++j) a[j] = __fdiv_rn(a[j], fl);
-      }
-      if (writer) {
-        float* o = p.out + (int64_t)(b0 + cur.bi) * p.out_ld + s.col_off + c * E + off;
-        if (p.flags & 2u) {
-          if constexpr (NF >= 4) {
-#pragma unroll
-            for (int j = 0; j < NF; j += 4)
-              __stcs(reinterpret_cast<float4*>(o + j), make_float4(a[j], a[j + 1], a[j + 2], a[j + 3]));
-          } else if constexpr (NF == 2) {
-            __stcs(reinterpret_cast<float2*>(o), make_float2(a[0], a[1]));
-          } else {
-            __stcs(o, a[0]);
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < NF; ++j) __stcs(o + j, a[j]);
-        }
-      }
+  for (int j = 0; j < N; ++j) {
+    float wj = 1.f;
+    if constexpr (PRED) {
+      if (wsum && j < left) wj = sw[j * GG];
+    } else if constexpr (WS) {
+      wj = sw[j * GG];
     }
-    if (!more) break;
-    cur = nxt;
-    qb = nqb;
-    base = nbase;
-    id_c = id_n;
-    w_c = w_n;
+    accumulate<DT>(acc, v[j], wj);
   }
 }
 
+// The steps that every lane of the warp has, without predicates, in batches of U, then 4, 2, 1.
+template <int DT, int GG, bool IND, bool WS>
+__device__ __forceinline__ int run_common(const uint32_t* srow, const float* sw, const RowAddr<IND>& ra,
+                                          int min_steps, unsigned long long* acc) {
+  constexpr int U = MFET_BAG_U;
+  int t = 0;
+  for (; t + U <= min_steps; t += U)
+    run_steps<DT, GG, IND, U, false, WS>(srow + t * GG, nullptr, sw + t * GG, ra, WS, 0, true, acc);
+  if constexpr (U > 4) {
+    if (t + 4 <= min_steps) {
+      run_steps<DT, GG, IND, 4, false, WS>(srow + t * GG, nullptr, sw + t * GG, ra, WS, 0, true, acc);
+      t += 4;
+    }
+  }
+  if constexpr (U > 2) {
+    if (t + 2 <= min_steps) {
+      run_steps<DT, GG, IND, 2, false, WS>(srow + t * GG, nullptr, sw + t * GG, ra, WS, 0, true, acc);
+      t += 2;
+    }
+  }
+  if (t < min_steps) {
+    run_steps<DT, GG, IND, 1, false, WS>(srow + t * GG, nullptr, sw + t * GG, ra, WS, 0, true, acc);
+    t += 1;
+  }
+  return t;
+}
 
-#define MFET_POOL_ARGS p, s, soff, b0, perm, ip, feat_lo
-
-// Bags perm[0 .. n_long) are long: one warp each. The rest: one row group each.
-template <int DT, int LPR, bool IND>
-__device__ __forceinline__ void pool_tile_lpr(const BagParams& p, const SlotDev& s, const int64_t* soff,
-                                              int b0, const uint8_t* perm, const IndirectParams& ip,
-                                              int64_t feat_lo, int n_long, int nb) {
-  if constexpr (LPR == 32) {
-    pool_tile<DT, 32, 32, IND>(p, s, soff, b0, perm, 0, nb, ip, feat_lo);
+// One bag piece per bag group of GG row groups: the staged rows pos0 + sub,
+// pos0 + sub + GG, ... below pos0 + len are added to acc. GG == 1: every row
+// group of the warp has its own (pos0, len); GG > 1: the warp shares them.
+// The steps that every lane of the warp has run without predicates; the few
+// that only some lanes have (the bags of a warp are of nearly the same length)
+// run predicated.
+template <int DT, int LPR, int GG, bool IND>
+__device__ __forceinline__ void gather_piece(const Win& w, const RowAddr<IND>& ra, int pos0, int len, int sub,
+                                             bool fast_ok, bool chunk_ok, bool wsum, unsigned long long* acc) {
+  // row loads (steps) of this lane, of the warp's busiest lane and of its idlest one
+  int steps, max_steps, min_steps;
+  if constexpr (GG == 1) {
+    steps = len;
+    max_steps = __reduce_max_sync(kFull, len);
+    min_steps = fast_ok ? __reduce_min_sync(kFull, len) : 0;
   } else {
-    if (n_long > 0) pool_tile<DT, LPR, 32, IND>(p, s, soff, b0, perm, 0, n_long, ip, feat_lo);
-    if (n_long < nb) pool_tile<DT, LPR, LPR, IND>(p, s, soff, b0, perm, n_long, nb, ip, feat_lo);
+    steps = (len - sub + GG - 1) / GG;
+    max_steps = (len + GG - 1) / GG;
+    min_steps = fast_ok ? len / GG : 0;
+  }
+  const uint32_t* srow = w.srow + pos0 + sub;
+  const uint32_t* shi = w.shi + pos0 + sub;
+  const float* sw = w.sw + pos0 + sub;
+  int t;
+  if (wsum) t = run_common<DT, GG, IND, true>(srow, sw, ra, min_steps, acc);
+  else t = run_common<DT, GG, IND, false>(srow, sw, ra, min_steps, acc);
+  if constexpr (GG == 1) {
+    for (; t < max_steps; t += 2)
+      run_steps<DT, GG, IND, 2, true, false>(srow + t * GG, shi + t * GG, sw + t * GG, ra, wsum, steps - t,
+                                             chunk_ok, acc);
+  } else {
+    // after the common steps at most one step is left, and not every row group has it
+    for (; t < max_steps; t += 1)
+      run_steps<DT, GG, IND, 1, true, false>(srow + t * GG, shi + t * GG, sw + t * GG, ra, wsum, steps - t,
+                                             chunk_ok, acc);
+  }
+}
+
+// Listed bag q of the window (or no bag: q < 0), pooled by a bag group of GG row
+// groups and stored (first piece), or added to what the earlier pieces left in
+// the output row.
+template <int DT, int LPR, int GG, bool IND>
+__device__ __forceinline__ void pool_bag(const BagParams& p, const SlotDev& s, const Win& w,
+                                         const RowAddr<IND>& ra, int q, int sub, int c, bool fast_ok,
+                                         bool chunk_ok, bool wsum) {
+  constexpr int E = ChunkElems<DT>::value;
+  constexpr int NF = (E / GG) > 0 ? (E / GG) : 1;  // values a lane stores
+  int pos0 = 0, len = 0, bag = -1;
+  if (q >= 0) {
+    pos0 = w.spos[q];
+    len = w.slen[q];
+    bag = w.sbag[q];
+  }
+  unsigned long long acc[E / 2];
+#pragma unroll
+  for (int j = 0; j < E / 2; ++j) acc[j] = 0ull;
+  gather_piece<DT, LPR, GG, IND>(w, ra, pos0, len, sub, fast_ok, chunk_ok, wsum, acc);
+
+  float a[E];
+#pragma unroll
+  for (int j = 0; j < E / 2; ++j) {
+    a[2 * j] = __uint_as_float((uint32_t)acc[j]);
+    a[2 * j + 1] = __uint_as_float((uint32_t)(acc[j] >> 32));
+  }
+  int off = 0;
+  bool writer = bag >= 0 && chunk_ok;
+  ReduceScatter<E, 0, GG, LPR>::run(a, sub, off, writer);
+  if (!writer) return;
+  const int bi = bag & 0xFF;
+  float* o = p.out + (int64_t)(w.b0 + bi) * p.out_ld + s.col_off + c * E + off;
+  if (bag & kNotFirst) {
+#pragma unroll
+    for (int j = 0; j < NF; ++j) a[j] += __ldcg(o + j);
+  }
+  if (s.pooling == MFET_POOL_MEAN && !(bag & kNotLast)) {
+    const int64_t blen = w.soff[bi + 1] - w.soff[bi];
+    if (blen > 0) {
+      const float inv = __frcp_rn((float)blen);  // correctly rounded reciprocal, then one rounding per product
+#pragma unroll
+      for (int j = 0; j < NF; ++j) a[j] *= inv;
+    }
+  }
+  if (p.flags & 2u) {
+    if constexpr (NF >= 4) {
+#pragma unroll
+      for (int j = 0; j < NF; j += 4)
+        __stcs(reinterpret_cast<float4*>(o + j), make_float4(a[j], a[j + 1], a[j + 2], a[j + 3]));
+    } else if constexpr (NF == 2) {
+      __stcs(reinterpret_cast<float2*>(o), make_float2(a[0], a[1]));
+    } else {
+      __stcs(o, a[0]);
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < NF; ++j) __stcs(o + j, a[j]);
+  }
+}
+
+// The warps of the block pool the window's bags: the long ones first, one warp
+// each, then the others, one row group each, handed out through the shared counter.
+template <int DT, int LPR, bool IND>
+__device__ __forceinline__ void pool_window(const BagParams& p, const SlotDev& s, const Win& w,
+                                            const IndirectParams& ip) {
+  constexpr int BPW = 32 / LPR;
+  const int lane = threadIdx.x & 31;
+  const int rg = lane / LPR;
+  const int c = lane & (LPR - 1);
+  const bool chunk_ok = c < (int)s.chunks;
+  const bool wsum = s.pooling == MFET_POOL_WSUM;
+  const bool fast_ok = (int)s.chunks == LPR && !(p.flags & 1u) && (IND || s.narrow != 0);
+  RowAddr<IND> ra;
+  const uint64_t coff = (uint64_t)c * ChunkElems<DT>::bytes;
+  if constexpr (IND) {
+    const uint64_t slot_off = reinterpret_cast<uint64_t>(s.table);  // byte offset of the column block in the row
+    ra.tbase = ip.cache_data + slot_off + coff;
+    ra.mbase = ip.cache_data + slot_off + s.meta_off;
+    ra.tbase2 = ip.staging + slot_off + coff;
+    ra.mbase2 = ip.staging + slot_off + s.meta_off;
+    ra.stride = ip.row_bytes;
+    ra.stride32 = (uint32_t)ip.row_bytes;
+    ra.wide = false;
+  } else {
+    ra.tbase = s.table + coff;
+    ra.mbase = s.table + s.meta_off;
+    ra.tbase2 = ra.mbase2 = nullptr;
+    ra.stride = s.stride;
+    ra.stride32 = (uint32_t)s.stride;
+    ra.wide = s.narrow == 0;
+  }
+  const int n_long = BPW > 1 ? w.n_long : 0;
+  while (true) {
+    int u = 0;
+    if (lane == 0) u = atomicAdd(w.next, 1);
+    u = __shfl_sync(kFull, u, 0);
+    if constexpr (BPW > 1) {
+      if (u < n_long) {
+        pool_bag<DT, LPR, BPW, IND>(p, s, w, ra, u, rg, c, fast_ok, chunk_ok, wsum);
+        continue;
+      }
+    }
+    const int q0 = n_long + (u - n_long) * BPW;
+    if (q0 >= w.nbw) break;
+    const int q = q0 + rg;
+    pool_bag<DT, LPR, 1, IND>(p, s, w, ra, q < w.nbw ? q : -1, 0, c, fast_ok, chunk_ok, wsum);
   }
 }
 
 template <int DT, bool IND>
-__device__ __forceinline__ void pool_tile_dt(const BagParams& p, const SlotDev& s, const int64_t* soff,
-                                             int b0, const uint8_t* perm, const IndirectParams& ip,
-                                             int64_t feat_lo, int n_long, int nb) {
+__device__ __forceinline__ void pool_window_dt(const BagParams& p, const SlotDev& s, const Win& w,
+                                               const IndirectParams& ip) {
   switch (s.lpr_log2) {
-    case 1: pool_tile_lpr<DT, 2, IND>(MFET_POOL_ARGS, n_long, nb); break;
-    case 2: pool_tile_lpr<DT, 4, IND>(MFET_POOL_ARGS, n_long, nb); break;
-    case 3: pool_tile_lpr<DT, 8, IND>(MFET_POOL_ARGS, n_long, nb); break;
-    case 4: pool_tile_lpr<DT, 16, IND>(MFET_POOL_ARGS, n_long, nb); break;
-    default: pool_tile_lpr<DT, 32, IND>(MFET_POOL_ARGS, n_long, nb); break;
+    case 1: pool_window<DT, 2, IND>(p, s, w, ip); break;
+    case 2: pool_window<DT, 4, IND>(p, s, w, ip); break;
+    case 3: pool_window<DT, 8, IND>(p, s, w, ip); break;
+    case 4: pool_window<DT, 16, IND>(p, s, w, ip); break;
+    default: pool_window<DT, 32, IND>(p, s, w, ip); break;
   }
 }
+
+// IDs (and weights) a thread requests before the tile's bags are ordered, so
+// that their latency overlaps the ordering.
+constexpr int kEarly = 4;
 
 // Q4 = true: the build of the kernel that also decodes INT4 rows (kept apart so that the
 // common kernels stay small).
 template <bool IND, bool Q4>
 __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParams& ip) {
+  extern __shared__ __align__(16) uint32_t dyn[];
   __shared__ int64_t soff[kMaxTile + 1];
   __shared__ int64_t sfeat[2];
-  __shared__ uint8_t perm[kMaxTile];
+  __shared__ int spos[kMaxTile], slen[kMaxTile], sbag[kMaxTile];
   constexpr int kSortWarps = kMaxTile / 32;  // warps whose threads own one bag each in the ordering
-  __shared__ int scnt[kSortWarps][16];
+  constexpr int kCnt = kSortWarps * (kLongBag + 1);  // per sorting warp: bags of length 0 .. kLongBag-1, long bags
+  static_assert(kCnt <= 256, "one thread clears one counter");
+  __shared__ int scnt[kSortWarps][kLongBag + 1];
+  __shared__ int snext;
+  const int tid = threadIdx.x;
   const int slot = blockIdx.x / p.tiles_per_slot;
   const int tile = blockIdx.x - slot * p.tiles_per_slot;
   const SlotDev& s = p.slot[slot];
   const int b0 = tile * p.tile;
   const int nb = min(p.tile, p.batch - b0);
+  const int C = p.stage_cap;
+  uint32_t* srow = dyn;
+  float* sw = reinterpret_cast<float*>(dyn + ((p.flags & 4u) ? C : 0));
+  uint32_t* shi = dyn + ((p.flags & 8u) ? ((p.flags & 4u) ? 2 * C : C) : 0);
   const long long* offs = reinterpret_cast<const long long*>(p.offsets) + (int64_t)s.feature * p.batch;
-  if ((int)threadIdx.x <= nb) soff[threadIdx.x] = __ldcs(offs + b0 + threadIdx.x);
-  if (IND && threadIdx.x < 2) sfeat[threadIdx.x] = offs[threadIdx.x ? p.batch : 0];
-  if (threadIdx.x >= 128 && threadIdx.x < 128 + kSortWarps * 16) (&scnt[0][0])[threadIdx.x - 128] = 0;
+  if (tid <= nb) soff[tid] = __ldcs(offs + b0 + tid);
+  if (IND && tid < 2) sfeat[tid] = offs[tid ? p.batch : 0];
+  if (tid < kCnt) (&scnt[0][0])[tid] = 0;
+  if (tid == 255) snext = 0;
   __syncthreads();
   int64_t feat_lo = 0;
   if constexpr (IND) {
@@ -389,54 +469,158 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
     const int64_t n_feat = sfeat[1] - sfeat[0];
     if (n_feat < 0 || n_feat > ip.cap) {
       __syncthreads();
-      if ((int)threadIdx.x <= nb) soff[threadIdx.x] = feat_lo;
+      if (tid <= nb) soff[tid] = feat_lo;
       __syncthreads();
     }
   }
+  const int64_t t0 = soff[0];
+  int64_t n_tile = soff[nb] - t0;
+  if (n_tile < 0) {
+    if (tid == 0) atomicOr(p.err, (uint32_t)MFET_DEV_OFFSETS);
+    n_tile = 0;
+  }
+  const bool wsum = s.pooling == MFET_POOL_WSUM;
+  const bool pre = (p.flags & 1u) != 0;
+  const bool wide = !IND && s.narrow == 0;
+  const unsigned long long* ids = reinterpret_cast<const unsigned long long*>(p.ids);
 
-  // Order the tile's bags by falling length class (counting sort over 16 classes, stable
-  // inside a class): class 15 = long bags (a whole warp each), classes 0..14 = shorter ones
-  // in steps of kLongBag/15, so that the bag groups of one warp get bags of similar length.
-  const int lane_ = threadIdx.x & 31, warp_ = threadIdx.x >> 5;
-  bool have = false;
-  int cls = 0, in_warp = 0;
-  if (warp_ < kSortWarps) {  // threads 0..kMaxTile-1 own one bag each
-    have = (int)threadIdx.x < nb;
-    if (have) {
-      const int64_t l = soff[threadIdx.x + 1] - soff[threadIdx.x];
-      const int len = l < 0 ? 0 : (l > 0x7FFFFFFF ? 0x7FFFFFFF : (int)l);
-      cls = len >= kLongBag ? 15 : (len * 15) / kLongBag;
+  // the ID (IND: the position in the dedup list) of a lookup -> staged value of window position pos
+  auto stage = [&](int pos, uint64_t id) {
+    if constexpr (IND) {
+      srow[pos] = (uint32_t)__ldg(ip.src + (uint32_t)id);
+    } else {
+      uint64_t row = pre ? id : mod_rows(splitmix64(id ^ s.seed), s.rows, s.magic);
+      if (row >= s.rows) {
+        atomicOr(p.err, (uint32_t)MFET_DEV_ROW_RANGE);
+        row = ~0ULL;  // sentinel: no row
+      }
+      srow[pos] = (uint32_t)row;
+      if (wide) shi[pos] = (uint32_t)(row >> 32);
     }
-    const unsigned peers = __match_any_sync(kFull, have ? cls : 16 + lane_);
-    in_warp = __popc(peers & ((1u << lane_) - 1u));
-    if (have && in_warp == 0) scnt[warp_][cls] = __popc(peers);
-  }
-  __syncthreads();
-  if (have) {
-    int rank = in_warp;
-    for (int w2 = 0; w2 < warp_; ++w2) rank += scnt[w2][cls];
-    for (int c2 = cls + 1; c2 < 16; ++c2)
-#pragma unroll
-      for (int w2 = 0; w2 < kSortWarps; ++w2) rank += scnt[w2][c2];
-    perm[rank] = (uint8_t)threadIdx.x;
-  }
-  __syncthreads();
-  int n_long = 0;
-#pragma unroll
-  for (int w2 = 0; w2 < kSortWarps; ++w2) n_long += scnt[w2][15];
-  if (p.group_policy == 1) n_long = 0;
-  if (p.group_policy == 2) n_long = nb;
+  };
+  auto fetch_id = [&](int64_t i) -> uint64_t {
+    if constexpr (IND) return (uint32_t)__ldg(ip.inverse + (i - feat_lo));
+    else return __ldcs(ids + i);
+  };
 
-  if constexpr (Q4) {
-    if (s.dtype == MFET_INT4) {
-      pool_tile_dt<MFET_INT4, IND>(MFET_POOL_ARGS, n_long, nb);
-      return;
+  for (int64_t w0 = 0;; w0 += C) {
+    const int wn = (int)(n_tile - w0 < (int64_t)C ? n_tile - w0 : (int64_t)C);
+    const int64_t g0 = t0 + w0;  // global index of window position 0
+    // ---- request the first IDs of the window --------------------------------
+    uint64_t eid[kEarly];
+    float ew[kEarly];
+#pragma unroll
+    for (int k = 0; k < kEarly; ++k) {
+      const int pos = tid + k * 256;
+      eid[k] = 0;
+      ew[k] = 1.f;
+      if (pos < wn) {
+        eid[k] = fetch_id(g0 + pos);
+        if (wsum) ew[k] = __ldcs(p.weights + g0 + pos);
+      }
     }
-  }
-  switch (s.dtype) {
-    case MFET_F32: pool_tile_dt<MFET_F32, IND>(MFET_POOL_ARGS, n_long, nb); break;
-    case MFET_F16: pool_tile_dt<MFET_F16, IND>(MFET_POOL_ARGS, n_long, nb); break;
-    default: pool_tile_dt<MFET_BF16, IND>(MFET_POOL_ARGS, n_long, nb); break;
+    // ---- order the bags that have a piece in this window: the long pieces first (a whole
+    // warp each), then the others by falling length (counting sort, stable among equal
+    // lengths), so that the row groups of one warp get pieces of nearly the same length.
+    // Empty bags belong to window 0.
+    const int lane_ = tid & 31, warp_ = tid >> 5;
+    bool have = false;
+    int cls = 0, in_warp = 0, plen = 0, ppos = 0, pbag = tid;
+    if (warp_ < kSortWarps) {  // threads 0..kMaxTile-1 own one bag each
+      if (tid < nb) {
+        const int64_t lo = soff[tid] - t0;
+        int64_t hi = soff[tid + 1] - t0;
+        if (hi < lo) {
+          if (w0 == 0) atomicOr(p.err, (uint32_t)MFET_DEV_OFFSETS);
+          hi = lo;
+        }
+        const int64_t a = lo > w0 ? lo : w0;
+        const int64_t b = hi < w0 + wn ? hi : w0 + wn;
+        if (b > a) {
+          plen = (int)(b - a);
+          ppos = (int)(a - w0);
+        }
+        have = plen > 0 || (w0 == 0 && hi == lo);
+        if (lo < w0 && w0 != 0) pbag |= kNotFirst;
+        if (hi > w0 + wn) pbag |= kNotLast;
+        cls = plen < kLongBag ? plen : kLongBag;
+      }
+      const unsigned peers = __match_any_sync(kFull, have ? cls : 64 + lane_);
+      in_warp = __popc(peers & ((1u << lane_) - 1u));
+      if (have && in_warp == 0) scnt[warp_][cls] = __popc(peers);
+    }
+    const int nbw = __syncthreads_count(have);
+    int n_long = 0;
+#pragma unroll
+    for (int w2 = 0; w2 < kSortWarps; ++w2) n_long += scnt[w2][kLongBag];
+    if (warp_ < kSortWarps) {
+      // lane c of every sorting warp: the bags of length c in all warps, and in the warps before this one
+      int tot = 0, before = 0, before_long = 0;
+      if (lane_ < kLongBag) {
+#pragma unroll
+        for (int w2 = 0; w2 < kSortWarps; ++w2) {
+          const int n = scnt[w2][lane_];
+          tot += n;
+          before += w2 < warp_ ? n : 0;
+        }
+      }
+#pragma unroll
+      for (int w2 = 0; w2 < kSortWarps; ++w2) before_long += w2 < warp_ ? scnt[w2][kLongBag] : 0;
+      // bags longer than c (and shorter than kLongBag): suffix sum over the lanes
+      int longer = tot;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_down_sync(kFull, longer, d);
+        if (lane_ + d < 32) longer += o;
+      }
+      const int start = n_long + longer - tot + before;  // first listed position of this warp's bags of length c
+      int rank = __shfl_sync(kFull, start, cls & 31);
+      if (cls == kLongBag) rank = before_long;
+      if (have) {
+        rank += in_warp;
+        spos[rank] = ppos;
+        slen[rank] = plen;
+        sbag[rank] = pbag;
+      }
+    }
+    // ---- hash the window's IDs into the staging buffer ------------------------
+#pragma unroll
+    for (int k = 0; k < kEarly; ++k) {
+      const int pos = tid + k * 256;
+      if (pos < wn) {
+        stage(pos, eid[k]);
+        if (wsum) sw[pos] = ew[k];
+      }
+    }
+    for (int pos = tid + kEarly * 256; pos < wn; pos += 256) {
+      stage(pos, fetch_id(g0 + pos));
+      if (wsum) sw[pos] = __ldcs(p.weights + g0 + pos);
+    }
+    __syncthreads();
+    if (p.group_policy == 1) n_long = 0;
+    if (p.group_policy == 2) n_long = nbw;
+
+    const Win w{srow, shi, sw, spos, slen, sbag, &snext, soff, nbw, n_long, b0};
+    bool done = false;
+    if constexpr (Q4) {
+      if (s.dtype == MFET_INT4) {
+        pool_window_dt<MFET_INT4, IND>(p, s, w, ip);
+        done = true;
+      }
+    }
+    if (!done) {
+      switch (s.dtype) {
+        case MFET_F32: pool_window_dt<MFET_F32, IND>(p, s, w, ip); break;
+        case MFET_F16: pool_window_dt<MFET_F16, IND>(p, s, w, ip); break;
+        default: pool_window_dt<MFET_BF16, IND>(p, s, w, ip); break;
+      }
+    }
+    if (w0 + C >= n_tile) break;
+    // ---- another window: everyone is done with the staging buffer and the bag list
+    __syncthreads();
+    if (tid < kCnt) (&scnt[0][0])[tid] = 0;
+    if (tid == 255) snext = 0;
+    __syncthreads();
   }
 }
 
@@ -468,19 +652,69 @@ static bool any_int4(const BagParams& p) {
   return false;
 }
 
-cudaError_t launch_bag_indirect(const BagParams& p, const IndirectParams& ip, cudaStream_t s) {
+// Dynamic shared memory of a launch: the staged row indices, plus the weights when a
+// slot is weighted, plus the upper index halves when a table needs them. Sets the
+// matching flag bits (4: weights staged, 8: upper halves staged).
+static size_t stage_bytes(BagParams& p, bool indirect) {
+  bool w = false, wide = false;
+  for (int i = 0; i < p.n_slots; ++i) {
+    w |= p.slot[i].pooling == MFET_POOL_WSUM;
+    wide |= !indirect && p.slot[i].narrow == 0;
+  }
+  p.flags &= ~12u;
+  if (w) p.flags |= 4u;
+  if (wide) p.flags |= 8u;
+  if (p.stage_cap < 32) p.stage_cap = kStageDefault;
+  if (p.stage_cap > kStageMax) p.stage_cap = kStageMax;
+  return (size_t)p.stage_cap * 4u * (1u + (w ? 1u : 0u) + (wide ? 1u : 0u));
+}
+
+// Shared-memory set-up of a kernel for a launch with `smem` dynamic bytes, redone only when
+// that size changes (per kernel and device): the opt-in above 48 KB, and a carve-out of just
+// what the resident blocks need, so that the rest of the SM's array stays L1 for the rows.
+template <typename K>
+static void prepare(K kernel, int which, size_t smem) {
+  static std::atomic<long long> configured[4][64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  const long long want = (long long)smem + 1;
+  if (configured[which][dev].load(std::memory_order_relaxed) == want) return;
+  if (smem > 48 * 1024) cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStageMax * 12);
+  const size_t per_block = smem + 4096 + 1024;  // dynamic + static + the system's share
+  size_t pct = (MFET_BAG_MINB * per_block * 100 + 228 * 1024 - 1) / (228 * 1024);
+  if (pct > 100) pct = 100;
+  cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)pct);
+  cudaGetLastError();
+  configured[which][dev].store(want, std::memory_order_relaxed);
+}
+
+cudaError_t launch_bag_indirect(const BagParams& p_, const IndirectParams& ip, cudaStream_t s) {
+  BagParams p = p_;
   const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
   if (blocks == 0) return cudaSuccess;
-  if (any_int4(p)) bag_indirect_q4_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, ip);
-  else bag_indirect_kernel<<<(unsigned)blocks, 256, 0, s>>>(p, ip);
+  const size_t smem = stage_bytes(p, true);
+  if (any_int4(p)) {
+    prepare(bag_indirect_q4_kernel, 0, smem);
+    bag_indirect_q4_kernel<<<(unsigned)blocks, 256, smem, s>>>(p, ip);
+  } else {
+    prepare(bag_indirect_kernel, 1, smem);
+    bag_indirect_kernel<<<(unsigned)blocks, 256, smem, s>>>(p, ip);
+  }
   return cudaGetLastError();
 }
 
-cudaError_t launch_bag(const BagParams& p, cudaStream_t s) {
+cudaError_t launch_bag(const BagParams& p_, cudaStream_t s) {
+  BagParams p = p_;
   const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
   if (blocks == 0) return cudaSuccess;
-  if (any_int4(p)) bag_q4_kernel<<<(unsigned)blocks, 256, 0, s>>>(p);
-  else bag_kernel<<<(unsigned)blocks, 256, 0, s>>>(p);
+  const size_t smem = stage_bytes(p, false);
+  if (any_int4(p)) {
+    prepare(bag_q4_kernel, 2, smem);
+    bag_q4_kernel<<<(unsigned)blocks, 256, smem, s>>>(p);
+  } else {
+    prepare(bag_kernel, 3, smem);
+    bag_kernel<<<(unsigned)blocks, 256, smem, s>>>(p);
+  }
   return cudaGetLastError();
 }
 

@@ -54,6 +54,7 @@ struct mfet_tables {
   uint64_t version = 0;  // caller's tag of this table set (model version)
   uint64_t prefetched = 0, consumed = 0;  // batches handed to mfet_host_prefetch / pooled from a prefetch
   int32_t tile = 0;  // bags per block; 0 = chosen from the batch size
+  int32_t stage_cap = 0;  // IDs staged per window of the pooling kernel; 0 = default
   int32_t profile = 0;             // 1: time the stages of the host-table path with events
   cudaEvent_t prof_ev[4] = {nullptr, nullptr, nullptr, nullptr};
   bool prof_valid = false;
@@ -77,7 +78,7 @@ struct SlotDev {
   uint8_t dtype;
   uint8_t pooling;
   uint8_t lpr_log2;      // lanes per row = 1 << lpr_log2 >= chunks
-  uint8_t narrow;        // 1: (rows*stride)/16 fits 32 bits
+  uint8_t narrow;        // 1: row indices and the stride fit 32 bits
   uint16_t pad;
   uint32_t meta_off;     // INT4: byte offset of the row's fp16 scale/bias pair from `table`
 };
@@ -85,6 +86,10 @@ static_assert(sizeof(SlotDev) == 64, "SlotDev must stay 64 bytes");
 
 constexpr int kMaxSlotsPerLaunch = 56;
 constexpr int kMaxTile = 128;
+// IDs of a tile that the pooling kernel stages in shared memory at a time
+// (4 bytes each, 8 with weights, 12 with weights and 64-bit row indices).
+constexpr int kStageDefault = 2048;
+constexpr int kStageMax = 8192;
 
 struct BagParams {
   const uint64_t* ids;
@@ -97,8 +102,11 @@ struct BagParams {
   int32_t n_slots;
   int32_t tiles_per_slot;
   int32_t tile;          // bags per block, <= kMaxTile
-  uint32_t flags;        // bit0: ids are rows; bit1: out allows 16-byte vector stores
+  uint32_t flags;        // bit0: ids are rows; bit1: out allows 16-byte vector stores;
+                         // set at launch: bit2 weights are staged, bit3 upper row-index halves are staged
   int32_t group_policy;  // 0 auto, 1 one row-group per bag, 2 one warp per bag
+  int32_t stage_cap;     // IDs staged per window, 32 .. kStageMax (0: default)
+  int32_t pad_;
   SlotDev slot[kMaxSlotsPerLaunch];
 };
 static_assert(sizeof(BagParams) <= 4000, "BagParams must fit the kernel parameter space");
