@@ -301,6 +301,13 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
     if args.alpha is not None:  # e.g. 0 = uniform IDs: no row repeats, the pure random-gather case
         w.alpha = np.full(w.n_features, float(args.alpha))
         w.name += ", Zipf alpha overridden to %g" % args.alpha
+    if args.device_slots_only:  # the HBM-resident part of a hybrid workload, as a workload of its own
+        keep = [s for s in range(w.n_slots) if w.tables[int(w.table_ids[s])].location == gi.LOC_DEVICE]
+        for t in w.tables:
+            if t.location != gi.LOC_DEVICE:
+                t.rows = 1024
+        w.slot_feature, w.table_ids, w.pooling = w.slot_feature[keep], w.table_ids[keep], w.pooling[keep]
+        w.name += ", device-table slots only"
     scaled_host = False
     fits = host_rows_that_fit(w)
     if fits:
@@ -319,7 +326,7 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
     if args.stage_ids:
         m.mfet_set_option(eng.h, m.OPT_STAGE_IDS, args.stage_ids)
     stream = torch.cuda.current_stream()
-    host_tabs = eng.host_table_ids()
+    host_tabs = [] if args.device_slots_only else eng.host_table_ids()
     cached_rows = 0
     B = w.batch
     host_feats = sorted({int(w.slot_feature[s]) for s in range(w.n_slots) if int(w.table_ids[s]) in host_tabs})
@@ -544,6 +551,8 @@ def main():
     ap.add_argument("--batches", type=int, default=8, help="distinct batches rotated through")
     ap.add_argument("--load-seconds", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--device-slots-only", action="store_true",
+                    help="drop the host-table slots of the workload (times the HBM-resident part of workload 5 alone)")
     ap.add_argument("--tile", type=int, default=0, help="samples per block of the pooling kernel (0 = library default)")
     ap.add_argument("--stage-ids", type=int, default=0, help="IDs staged per pass of the pooling kernel (0 = library default)")
     args = ap.parse_args()

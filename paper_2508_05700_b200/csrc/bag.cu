@@ -242,7 +242,8 @@ __device__ __forceinline__ void run_steps(const uint32_t* srow, const uint32_t* 
   }
 }
 
-// The steps that every lane of the warp has, without predicates, in batches of U, then 4, 2, 1.
+// The steps that every lane of the warp has, without predicates, in batches of U, then 4;
+// up to 3 of them are left to the predicated batches.
 template <int DT, int GG, bool IND, bool WS>
 __device__ __forceinline__ int run_common(const uint32_t* srow, const float* sw, const RowAddr<IND>& ra,
                                           int min_steps, unsigned long long* acc) {
@@ -256,25 +257,16 @@ __device__ __forceinline__ int run_common(const uint32_t* srow, const float* sw,
       t += 4;
     }
   }
-  if constexpr (U > 2) {
-    if (t + 2 <= min_steps) {
-      run_steps<DT, GG, IND, 2, false, WS>(srow + t * GG, nullptr, sw + t * GG, ra, WS, 0, true, acc);
-      t += 2;
-    }
-  }
-  if (t < min_steps) {
-    run_steps<DT, GG, IND, 1, false, WS>(srow + t * GG, nullptr, sw + t * GG, ra, WS, 0, true, acc);
-    t += 1;
-  }
   return t;
 }
 
 // One bag piece per bag group of GG row groups: the staged rows pos0 + sub,
 // pos0 + sub + GG, ... below pos0 + len are added to acc. GG == 1: every row
 // group of the warp has its own (pos0, len); GG > 1: the warp shares them.
-// The steps that every lane of the warp has run without predicates; the few
-// that only some lanes have (the bags of a warp are of nearly the same length)
-// run predicated.
+// The steps that every lane of the warp has run without predicates in batches
+// of U and 4; the last few, and those that only some lanes have (the bags of a
+// warp are of nearly the same length), run in predicated batches of 4: every
+// batch is one round trip to memory, so the remainder is not split further.
 template <int DT, int LPR, int GG, bool IND>
 __device__ __forceinline__ void gather_piece(const Win& w, const RowAddr<IND>& ra, int pos0, int len, int sub,
                                              bool fast_ok, bool chunk_ok, bool wsum, unsigned long long* acc) {
@@ -295,16 +287,10 @@ __device__ __forceinline__ void gather_piece(const Win& w, const RowAddr<IND>& r
   int t;
   if (wsum) t = run_common<DT, GG, IND, true>(srow, sw, ra, min_steps, acc);
   else t = run_common<DT, GG, IND, false>(srow, sw, ra, min_steps, acc);
-  if constexpr (GG == 1) {
-    for (; t < max_steps; t += 2)
-      run_steps<DT, GG, IND, 2, true, false>(srow + t * GG, shi + t * GG, sw + t * GG, ra, wsum, steps - t,
-                                             chunk_ok, acc);
-  } else {
-    // after the common steps at most one step is left, and not every row group has it
-    for (; t < max_steps; t += 1)
-      run_steps<DT, GG, IND, 1, true, false>(srow + t * GG, shi + t * GG, sw + t * GG, ra, wsum, steps - t,
-                                             chunk_ok, acc);
-  }
+  // what is left: fewer than 4 common steps and the steps that only some lanes have
+  for (; t < max_steps; t += 4)
+    run_steps<DT, GG, IND, 4, true, false>(srow + t * GG, shi + t * GG, sw + t * GG, ra, wsum, steps - t, chunk_ok,
+                                           acc);
 }
 
 // Listed bag q of the window (or no bag: q < 0), pooled by a bag group of GG row

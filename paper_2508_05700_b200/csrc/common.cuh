@@ -106,7 +106,6 @@ struct BagParams {
                          // set at launch: bit2 weights are staged, bit3 upper row-index halves are staged
   int32_t group_policy;  // 0 auto, 1 one row-group per bag, 2 one warp per bag
   int32_t stage_cap;     // IDs staged per window, 32 .. kStageMax (0: default)
-  int32_t pad_;
   SlotDev slot[kMaxSlotsPerLaunch];
 };
 static_assert(sizeof(BagParams) <= 4000, "BagParams must fit the kernel parameter space");
