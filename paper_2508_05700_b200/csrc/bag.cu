@@ -37,7 +37,7 @@
 #define MFET_BAG_U 8
 #endif
 #ifndef MFET_BAG_LONG
-#define MFET_BAG_LONG 32
+#define MFET_BAG_LONG 64
 #endif
 #ifndef MFET_BAG_MINB
 #define MFET_BAG_MINB 4
@@ -49,7 +49,10 @@ namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
 constexpr int kLongBag = MFET_BAG_LONG;  // bags at least this long get a whole warp
-static_assert(kLongBag >= 1 && kLongBag <= 32, "the ordering has one lane per shorter length");
+// the ordering of the shorter bags has one lane per length class: classes of kClassW lengths
+constexpr int kClassW = (kLongBag + 31) / 32;
+constexpr int kClasses = (kLongBag + kClassW - 1) / kClassW;  // <= 32; class kClasses = long bags
+static_assert(kLongBag >= 1 && kClasses <= 32, "one lane per class of shorter bags");
 
 // A lane's piece of a row: 16 bytes (4 fp32 or 8 fp16/bf16 values), or for INT4 rows
 // 4 bytes (8 four-bit codes) plus the row's fp16 scale/bias pair.
@@ -427,9 +430,9 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   __shared__ int64_t sfeat[2];
   __shared__ int spos[kMaxTile], slen[kMaxTile], sbag[kMaxTile];
   constexpr int kSortWarps = kMaxTile / 32;  // warps whose threads own one bag each in the ordering
-  constexpr int kCnt = kSortWarps * (kLongBag + 1);  // per sorting warp: bags of length 0 .. kLongBag-1, long bags
+  constexpr int kCnt = kSortWarps * (kClasses + 1);  // per sorting warp: the classes of shorter bags, long bags
   static_assert(kCnt <= 256, "one thread clears one counter");
-  __shared__ int scnt[kSortWarps][kLongBag + 1];
+  __shared__ int scnt[kSortWarps][kClasses + 1];
   __shared__ int snext;
   const int tid = threadIdx.x;
   const int slot = blockIdx.x / p.tiles_per_slot;
@@ -506,8 +509,8 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
       }
     }
     // ---- order the bags that have a piece in this window: the long pieces first (a whole
-    // warp each), then the others by falling length (counting sort, stable among equal
-    // lengths), so that the row groups of one warp get pieces of nearly the same length.
+    // warp each), then the others by falling length class (counting sort, stable inside a
+    // class), so that the row groups of one warp get pieces of nearly the same length.
     // Empty bags belong to window 0.
     const int lane_ = tid & 31, warp_ = tid >> 5;
     bool have = false;
@@ -529,7 +532,7 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
         have = plen > 0 || (w0 == 0 && hi == lo);
         if (lo < w0 && w0 != 0) pbag |= kNotFirst;
         if (hi > w0 + wn) pbag |= kNotLast;
-        cls = plen < kLongBag ? plen : kLongBag;
+        cls = plen < kLongBag ? plen / kClassW : kClasses;
       }
       const unsigned peers = __match_any_sync(kFull, have ? cls : 64 + lane_);
       in_warp = __popc(peers & ((1u << lane_) - 1u));
@@ -538,11 +541,11 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
     const int nbw = __syncthreads_count(have);
     int n_long = 0;
 #pragma unroll
-    for (int w2 = 0; w2 < kSortWarps; ++w2) n_long += scnt[w2][kLongBag];
+    for (int w2 = 0; w2 < kSortWarps; ++w2) n_long += scnt[w2][kClasses];
     if (warp_ < kSortWarps) {
-      // lane c of every sorting warp: the bags of length c in all warps, and in the warps before this one
+      // lane c of every sorting warp: the bags of class c in all warps, and in the warps before this one
       int tot = 0, before = 0, before_long = 0;
-      if (lane_ < kLongBag) {
+      if (lane_ < kClasses) {
 #pragma unroll
         for (int w2 = 0; w2 < kSortWarps; ++w2) {
           const int n = scnt[w2][lane_];
@@ -551,17 +554,17 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
         }
       }
 #pragma unroll
-      for (int w2 = 0; w2 < kSortWarps; ++w2) before_long += w2 < warp_ ? scnt[w2][kLongBag] : 0;
-      // bags longer than c (and shorter than kLongBag): suffix sum over the lanes
+      for (int w2 = 0; w2 < kSortWarps; ++w2) before_long += w2 < warp_ ? scnt[w2][kClasses] : 0;
+      // shorter bags of a higher class than c: suffix sum over the lanes
       int longer = tot;
 #pragma unroll
       for (int d = 1; d < 32; d <<= 1) {
         const int o = __shfl_down_sync(kFull, longer, d);
         if (lane_ + d < 32) longer += o;
       }
-      const int start = n_long + longer - tot + before;  // first listed position of this warp's bags of length c
+      const int start = n_long + longer - tot + before;  // first listed position of this warp's bags of class c
       int rank = __shfl_sync(kFull, start, cls & 31);
-      if (cls == kLongBag) rank = before_long;
+      if (cls == kClasses) rank = before_long;
       if (have) {
         rank += in_warp;
         spos[rank] = ppos;
@@ -666,7 +669,9 @@ static void prepare(K kernel, int which, size_t smem) {
   const long long want = (long long)smem + 1;
   if (configured[which][dev].load(std::memory_order_relaxed) == want) return;
   if (smem > 48 * 1024) cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStageMax * 12);
-  const size_t per_block = smem + 4096 + 1024;  // dynamic + static + the system's share
+  cudaFuncAttributes fa{};
+  if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) fa.sharedSizeBytes = 4096;
+  const size_t per_block = smem + fa.sharedSizeBytes + 1024;  // dynamic + static + the system's share
   size_t pct = (MFET_BAG_MINB * per_block * 100 + 228 * 1024 - 1) / (228 * 1024);
   if (pct > 100) pct = 100;
   cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)pct);

@@ -215,6 +215,52 @@ def test_unit_parity(dtype, dim, pattern, policy):
         mt.close()
 
 
+@pytest.mark.parametrize("stage", [32, 100, 2048])
+@pytest.mark.parametrize("tile", [8, 32, 128])
+@pytest.mark.parametrize("dtype,dim", [(gi.BF16, 64), (gi.F16, 32), (gi.F32, 128), (gi.BF16, 24)])
+def test_staging_windows_cut_bags_anywhere(stage, tile, dtype, dim):
+    """A tile with more IDs than the staging capacity is pooled in several passes: bags cut by a
+    pass boundary (once or many times), empty bags on a boundary and tiles that end on one give
+    the oracle's result for every pooling, whatever the capacity and the tile size."""
+    rng = np.random.default_rng(stage * 131 + tile * 7 + dim)
+    B = 150
+    lens = rng.integers(0, 40, size=B)
+    lens[rng.random(B) < 0.2] = 0
+    # bags that fill whole passes (at most 700 IDs: the fp32 tolerance is derived for bags of that size)
+    lens[[3, 77, 149]] = [min(stage, 600), min(3 * stage + 5, 700), min(2 * stage, 650)]
+    lens[[4, 5]] = 0  # empty bags right behind one
+    off = np.zeros(B + 1, np.int64)
+    np.cumsum(lens, out=off[1:])
+    tab = (0.01 * rng.standard_normal((211, dim))).astype(np.float32)
+    mt = _Mat([tab], [dtype], seeds=[0x5EED])
+    try:
+        mt.m.mfet_set_option(mt.h, mt.m.OPT_TILE, tile)
+        mt.m.mfet_set_option(mt.h, mt.m.OPT_STAGE_IDS, stage)
+        ids = rng.integers(0, 2**40, size=int(off[-1]), dtype=np.uint64)
+        w = rng.random(ids.size).astype(np.float32)
+        for pool in (0, 1, 2):
+            got = forward(mt, B, 1, [0], [0], [pool], ids, off, w)
+            ref = orc.embedding_bag(mt.oracle_tables, B, 1, [0], [0], [pool], ids, off, w)
+            assert_close(got, ref, "pool %d" % pool)
+            assert not got[lens == 0].any()
+        assert mt.m.mfet_query_status(mt.h, clear=True) == 0
+    finally:
+        mt.close()
+
+
+def test_stage_option_range():
+    mt = _Mat([np.zeros((4, 8), np.float32)], [gi.F32])
+    try:
+        m = mt.m
+        for bad in (1, 31, 8193, -5):
+            with pytest.raises(m.MfetError):
+                m.mfet_set_option(mt.h, m.OPT_STAGE_IDS, bad)
+        for good in (0, 32, 8192):
+            m.mfet_set_option(mt.h, m.OPT_STAGE_IDS, good)
+    finally:
+        mt.close()
+
+
 def test_single_row_table_and_prehashed_rows():
     rng = np.random.default_rng(3)
     tab = rng.standard_normal((1, 32)).astype(np.float32)
@@ -398,6 +444,9 @@ def test_host_table_path_matches_oracle_and_hbm_placement(pinned_by_caller):
         assert_close(workload_forward(dt, w, b1), workload_oracle(dt, w, b1), "host path, cache on")
         dt.build_cache(0, np.arange(0, w.tables[0].rows, dtype=np.int64))  # everything cached
         assert np.array_equal(workload_forward(dt, w, b), cold)
+        dt.m.mfet_set_option(dt.h, dt.m.OPT_STAGE_IDS, 96)  # many staging passes per tile, bags cut between them
+        assert_close(workload_forward(dt, w, b), ref, "host path, small staging buffer")
+        dt.m.mfet_set_option(dt.h, dt.m.OPT_STAGE_IDS, 0)
         launches = dt.m.mfet_launch_count(dt.h)
         assert launches > 0
     # the same table placed in HBM gives the same bits
