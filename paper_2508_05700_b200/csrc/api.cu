@@ -96,7 +96,11 @@ int mfet_tables_create(const mfet_table_desc_t* descs, int32_t n_tables, int32_t
     *h->err_host = 0;
     ok = cudaHostGetDevicePointer((void**)&h->err_dev, h->err_host, 0) == cudaSuccess;
   }
-  ok = ok && cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) == cudaSuccess;
+  // host-table slots are the long pole of a hybrid batch (their rows cross PCIe), so their
+  // kernels get the SMs first when they compete with the pooling of the device tables
+  int prio_lo = 0, prio_hi = 0;
+  ok = ok && cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
