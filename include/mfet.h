@@ -307,10 +307,10 @@ MFET_API int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits /*h
  * bags: 0 = a bag of 64 or more IDs gets a whole warp, a shorter one the lanes that
  * cover one row (default), 1 = one row's lanes for every bag, 2 = a warp for every
  * bag. The result is the same up to the order of fp32 additions. MFET_OPT_TILE:
- * samples per thread block of the pooling kernel: 0 = chosen from the batch size
- * (default), or 8 .. 128 (multiples of 32 suit the kernel best). MFET_OPT_STAGE_IDS:
+ * samples per thread block of the pooling kernel: 0 = chosen per launch so that the
+ * blocks fill the SMs evenly (default), or 8 .. 128. MFET_OPT_STAGE_IDS:
  * how many IDs of a tile the pooling kernel hashes into shared memory at a time:
- * 0 = default (2048, or 4096 with 128-sample tiles), or 32 .. 8192; a tile with more
+ * 0 = default (4096), or 32 .. 8192; a tile with more
  * IDs is pooled in several passes and a bag cut by a pass boundary continues from
  * its partial sum (same result up to the order of fp32 additions). MFET_OPT_PROFILE:
  * 1 = record CUDA events around the stages of the host-table path of every forward

@@ -382,13 +382,9 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
   p.flags = (uint32_t)(shape->flags & 1);
   if (aligned16(out) && out_ld % 4 == 0) p.flags |= 2u;
   p.group_policy = t->group_policy;
-  // bags per block: full tiles once there is enough work to fill the GPU several times over
-  const int64_t bags = (int64_t)B * L;
-  p.tile = bags >= 148LL * 16 * 128 ? 128 : (bags >= 16384 ? 64 : (bags >= 4096 ? 32 : 16));
-  if (t->tile) p.tile = t->tile;
-  // staging capacity: room for the IDs of a typical tile (a tile with more is pooled in several passes)
-  p.stage_cap = t->stage_cap ? t->stage_cap : (p.tile >= 128 ? 2 * kStageDefault : kStageDefault);
-  p.tiles_per_slot = (B + p.tile - 1) / p.tile;
+  // samples per block and staging capacity: the caller's options, else chosen at launch (0)
+  p.tile = t->tile;
+  p.stage_cap = t->stage_cap;
 
   // host-table slots go to the side stream, forked from and joined to `stream`
   bool forked = false;

@@ -26,7 +26,12 @@
 // sum that its earlier piece left in the output row. The order of additions
 // depends only on the inputs, the tile size and the staging capacity, never on
 // timing.
+#include <algorithm>
 #include <atomic>
+#include <functional>
+#include <mutex>
+#include <queue>
+#include <vector>
 
 #include "common.cuh"
 
@@ -641,9 +646,86 @@ static bool any_int4(const BagParams& p) {
   return false;
 }
 
-// Dynamic shared memory of a launch: the staged row indices, plus the weights when a
-// slot is weighted, plus the upper index halves when a table needs them. Sets the
-// matching flag bits (4: weights staged, 8: upper halves staged).
+// Samples per block when the caller has not fixed them. The blocks of a launch are handed to
+// the SMs in index order (slots with the widest rows first), kMinBlocks at a time per SM; a
+// block costs a fixed part (offsets, IDs, hashing, barriers) plus a part that grows with
+// samples x lanes per row. The launch ends when the last block does, so for grids of one or
+// two waves the tile decides how full the last wave is (4096 samples x 8 slots: 56-sample
+// tiles make exactly 592 blocks = one block slot each on 148 SMs, 64-sample tiles leave 80
+// slots idle and every block 14 % longer). For every candidate tile the order of dispatch is
+// played through on the host (a heap of block-slot free times) and the shortest wins; the
+// result is remembered per launch shape. When all slots have the same row width, only tiles
+// that fit one wave compete with the size-based default: equal blocks in two or more whole
+// waves run in lockstep (all hashing, then all gathering), which measured 5-8 % slower than a
+// ragged last wave. Large grids take full tiles without the exercise.
+static int choose_tile(const BagParams& p) {
+  constexpr double kFixed = 20.0;  // fixed cost of a block, in samples of a 128-byte-row slot
+  static std::mutex mu;
+  struct Entry { int dev, batch, n, cnt[8], tile; };
+  static std::vector<Entry> memo;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  static std::atomic<int> sm_count[64];
+  int sms = dev >= 0 && dev < 64 ? sm_count[dev].load(std::memory_order_relaxed) : 0;
+  if (sms == 0) {
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    if (dev >= 0 && dev < 64) sm_count[dev].store(sms, std::memory_order_relaxed);
+  }
+  const int slots = sms * MFET_BAG_MINB;
+  if ((int64_t)p.n_slots * ((p.batch + kMaxTile - 1) / kMaxTile) >= 6LL * slots) return kMaxTile;
+  Entry key{};
+  key.dev = dev;
+  key.batch = p.batch;
+  key.n = p.n_slots;
+  for (int i = 0; i < p.n_slots; ++i) key.cnt[p.slot[i].lpr_log2 & 7] += 1;
+  {
+    std::lock_guard<std::mutex> g(mu);
+    for (const Entry& e : memo)
+      if (e.dev == key.dev && e.batch == key.batch && e.n == key.n && std::equal(e.cnt, e.cnt + 8, key.cnt)) return e.tile;
+  }
+  bool same_width = true;
+  for (int i = 1; i < p.n_slots; ++i) same_width &= p.slot[i].lpr_log2 == p.slot[0].lpr_log2;
+  const int64_t bags = (int64_t)p.batch * p.n_slots;
+  const int by_size = bags >= 16384 ? 64 : (bags >= 4096 ? 32 : 16);
+  int best = by_size;
+  double best_t = 1e300;
+  for (int tile = kMaxTile; tile >= 16; tile -= 8) {
+    const int tiles = (p.batch + tile - 1) / tile;
+    if ((int64_t)tiles * p.n_slots > 8LL * slots) break;  // many waves: the tile no longer matters
+    if (same_width && (int64_t)tiles * p.n_slots > slots && tile != by_size) continue;
+    std::priority_queue<double, std::vector<double>, std::greater<double>> free_at;
+    double end = 0.0;
+    int running = 0;
+    for (int i = 0; i < p.n_slots; ++i) {
+      const double full = kFixed + tile * (double)(1 << p.slot[i].lpr_log2) / 8.0;
+      for (int k = 0; k < tiles; ++k) {
+        const int nb = std::min(tile, p.batch - k * tile);
+        const double cost = kFixed + (full - kFixed) * nb / tile;
+        double start = 0.0;
+        if (running < slots) {
+          ++running;
+        } else {
+          start = free_at.top();
+          free_at.pop();
+        }
+        free_at.push(start + cost);
+        end = std::max(end, start + cost);
+      }
+    }
+    if (end < best_t) {
+      best_t = end;
+      best = tile;
+    }
+  }
+  key.tile = best;
+  std::lock_guard<std::mutex> g(mu);
+  if (memo.size() < 256) memo.push_back(key);
+  return best;
+}
+
+// Tile, grid and dynamic shared memory of a launch: the staged row indices, plus the
+// weights when a slot is weighted, plus the upper index halves when a table needs them.
+// Sets the matching flag bits (4: weights staged, 8: upper halves staged).
 static size_t stage_bytes(BagParams& p, bool indirect) {
   bool w = false, wide = false;
   for (int i = 0; i < p.n_slots; ++i) {
@@ -653,6 +735,10 @@ static size_t stage_bytes(BagParams& p, bool indirect) {
   p.flags &= ~12u;
   if (w) p.flags |= 4u;
   if (wide) p.flags |= 8u;
+  if (p.tile <= 0) p.tile = choose_tile(p);
+  if (p.tile > kMaxTile) p.tile = kMaxTile;
+  p.tiles_per_slot = (p.batch + p.tile - 1) / p.tile;
+  // staging capacity: room for the IDs of a typical tile (a tile with more is pooled in several passes)
   if (p.stage_cap < 32) p.stage_cap = kStageDefault;
   if (p.stage_cap > kStageMax) p.stage_cap = kStageMax;
   return (size_t)p.stage_cap * 4u * (1u + (w ? 1u : 0u) + (wide ? 1u : 0u));
@@ -681,9 +767,9 @@ static void prepare(K kernel, int which, size_t smem) {
 
 cudaError_t launch_bag_indirect(const BagParams& p_, const IndirectParams& ip, cudaStream_t s) {
   BagParams p = p_;
-  const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
-  if (blocks == 0) return cudaSuccess;
+  if (p.n_slots == 0 || p.batch <= 0) return cudaSuccess;
   const size_t smem = stage_bytes(p, true);
+  const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
   if (any_int4(p)) {
     prepare(bag_indirect_q4_kernel, 0, smem);
     bag_indirect_q4_kernel<<<(unsigned)blocks, 256, smem, s>>>(p, ip);
@@ -696,9 +782,9 @@ cudaError_t launch_bag_indirect(const BagParams& p_, const IndirectParams& ip, c
 
 cudaError_t launch_bag(const BagParams& p_, cudaStream_t s) {
   BagParams p = p_;
-  const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
-  if (blocks == 0) return cudaSuccess;
+  if (p.n_slots == 0 || p.batch <= 0) return cudaSuccess;
   const size_t smem = stage_bytes(p, false);
+  const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
   if (any_int4(p)) {
     prepare(bag_q4_kernel, 2, smem);
     bag_q4_kernel<<<(unsigned)blocks, 256, smem, s>>>(p);

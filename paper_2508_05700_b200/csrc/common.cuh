@@ -88,7 +88,7 @@ constexpr int kMaxSlotsPerLaunch = 56;
 constexpr int kMaxTile = 128;
 // IDs of a tile that the pooling kernel stages in shared memory at a time
 // (4 bytes each, 8 with weights, 12 with weights and 64-bit row indices).
-constexpr int kStageDefault = 2048;
+constexpr int kStageDefault = 4096;
 constexpr int kStageMax = 8192;
 
 struct BagParams {
