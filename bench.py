@@ -470,6 +470,47 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
                          for k in range(n_rot)]))
     d2h = float(w.batch * w.out_dim * 4)
 
+    # ---- hashing alone and dedup alone (not part of the timed step) ----------
+    alone = None
+    if world == 1:
+        def timed(fn, reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(3):
+                fn()
+            a.record(stream)
+            for _ in range(reps):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps * 1e3  # us
+
+        s0 = 0
+        t0, f0 = int(w.table_ids[s0]), int(w.slot_feature[s0])
+        n_all = nnz[0]
+        rows_all = torch.empty(n_all, dtype=torch.int64, device="cuda")
+        us_hash = timed(lambda: m.mfet_hash_ids(eng.h, t0, d_ids[0], n_all, rows_all, stream.cuda_stream), 100)
+        n_big = 1 << 24
+        big = torch.randint(0, 1 << 40, (n_big,), dtype=torch.int64, device="cuda")
+        big_out = torch.empty_like(big)
+        us_big = timed(lambda: m.mfet_hash_ids(eng.h, t0, big, n_big, big_out, stream.cuda_stream), 20)
+        lo, hi = int(batches[0].offsets[f0 * B]), int(batches[0].offsets[(f0 + 1) * B])
+        n_f = hi - lo
+        if eng.ws is None:
+            eng.set_workspace(n_f + 1024)
+        m.mfet_hash_ids(eng.h, t0, d_ids[0][lo:hi], n_f, rows_all, stream.cuda_stream)
+        uniq = torch.empty(n_f, dtype=torch.int64, device="cuda")
+        inv = torch.empty(n_f, dtype=torch.int32, device="cuda")
+        n_uniq = torch.zeros(1, dtype=torch.int64, device="cuda")
+        us_dedup = timed(lambda: m.mfet_dedup_rows(eng.h, rows_all, n_f, uniq, inv, n_uniq, w.tables[t0].rows - 1,
+                                                   stream.cuda_stream), 50)
+        peak_bw, _ = measured_peaks()
+        alone = {"hash": {"ids": n_all, "us": us_hash, "ids_large": n_big, "us_large": us_big,
+                          "gbps_large": n_big * 16 / us_big / 1e3, "frac_large": n_big * 16 / us_big / 1e3 / peak_bw,
+                          "bytes_per_id": 16},
+                 "dedup": {"ids": n_f, "unique": int(n_uniq.item()), "us": us_dedup,
+                           "table_rows": int(w.tables[t0].rows)}}
+        del big, big_out, rows_all, uniq, inv
+
     ms, units = aggregate_over_ranks(local_ms, float(ids_done), dist if world > 1 else None)
     e2e_ms_all, _ = aggregate_over_ranks(e2e_ms, float(ids_done), dist if world > 1 else None)
     eng.close()
@@ -498,6 +539,7 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
                      "kernel": "bag_kernel (all HBM-resident slots, one launch)",
                      "algorithmic_bytes_per_launch": alg, "kernel_ms": kern_ms},
         "roofline_host_path": host_path,
+        "stages_alone": alone,
         "cpu_baseline": base,
         "clocks": clocks,
     }
@@ -527,7 +569,7 @@ def run_gpu(args):
         try:
             hyb = measure(args, 5, rank, world, dist, False, sampler_gpu=None)
             line["hybrid"] = {k: hyb[k] for k in ("value", "unit", "ms_per_step", "config", "e2e", "gpu_launches",
-                                                  "roofline", "roofline_host_path")}
+                                                  "roofline", "roofline_host_path", "stages_alone")}
         except Exception as exc:  # the headline number stands on its own
             line["hybrid"] = {"error": "%s: %s" % (type(exc).__name__, exc)}
     if world > 1:
