@@ -3,27 +3,58 @@
 
 namespace mfet {
 
-// rows_out[i] = splitmix64(ids[i] ^ seed) mod rows. One ID per thread,
-// grid-stride; 8-byte coalesced loads and stores, streaming hints (each value is
-// touched once).
+// rows_out[i] = splitmix64(ids[i] ^ seed) mod rows, grid-stride, streaming hints (each value
+// is touched once). PAIRS: a thread takes two neighbouring IDs with one 16-byte load and one
+// 16-byte store, two such pairs in flight (the arrays must be 16-byte aligned; an odd last ID
+// is left to the first thread). Otherwise one ID per thread and 8-byte accesses.
+template <bool PAIRS>
 __global__ void __launch_bounds__(256) hash_kernel(const uint64_t* __restrict__ ids, int64_t n,
                                                    uint64_t seed, uint64_t rows, uint64_t magic,
                                                    int64_t* __restrict__ rows_out) {
-  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t step = (int64_t)gridDim.x * blockDim.x;
-  for (; i < n; i += step) {
-    uint64_t id = __ldcs(reinterpret_cast<const unsigned long long*>(ids) + i);
-    uint64_t r = mod_rows(splitmix64(id ^ seed), rows, magic);
-    __stcs(reinterpret_cast<long long*>(rows_out) + i, (long long)r);
+  if constexpr (PAIRS) {
+    const int64_t np = n >> 1;
+    const ulonglong2* in2 = reinterpret_cast<const ulonglong2*>(ids);
+    longlong2* out2 = reinterpret_cast<longlong2*>(rows_out);
+    int64_t i = first;
+    for (; i + step < np; i += 2 * step) {
+      const ulonglong2 a = __ldcs(in2 + i), b = __ldcs(in2 + i + step);
+      longlong2 ra, rb;
+      ra.x = (long long)mod_rows(splitmix64(a.x ^ seed), rows, magic);
+      ra.y = (long long)mod_rows(splitmix64(a.y ^ seed), rows, magic);
+      rb.x = (long long)mod_rows(splitmix64(b.x ^ seed), rows, magic);
+      rb.y = (long long)mod_rows(splitmix64(b.y ^ seed), rows, magic);
+      __stcs(out2 + i, ra);
+      __stcs(out2 + i + step, rb);
+    }
+    if (i < np) {
+      const ulonglong2 a = __ldcs(in2 + i);
+      longlong2 ra;
+      ra.x = (long long)mod_rows(splitmix64(a.x ^ seed), rows, magic);
+      ra.y = (long long)mod_rows(splitmix64(a.y ^ seed), rows, magic);
+      __stcs(out2 + i, ra);
+    }
+    if ((n & 1) && first == 0)
+      rows_out[n - 1] = (int64_t)mod_rows(splitmix64(ids[n - 1] ^ seed), rows, magic);
+  } else {
+    for (int64_t i = first; i < n; i += step) {
+      uint64_t id = __ldcs(reinterpret_cast<const unsigned long long*>(ids) + i);
+      uint64_t r = mod_rows(splitmix64(id ^ seed), rows, magic);
+      __stcs(reinterpret_cast<long long*>(rows_out) + i, (long long)r);
+    }
   }
 }
 
 cudaError_t launch_hash(const uint64_t* ids, int64_t n, uint64_t seed, uint64_t rows, uint64_t magic,
                         int64_t* rows_out, cudaStream_t s) {
   if (n == 0) return cudaSuccess;
-  int64_t blocks = (n + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
-  hash_kernel<<<(unsigned)blocks, 256, 0, s>>>(ids, n, seed, rows, magic, rows_out);
+  const bool pairs = n >= 2 && ((reinterpret_cast<uintptr_t>(ids) | reinterpret_cast<uintptr_t>(rows_out)) & 15u) == 0;
+  const int64_t items = pairs ? (n >> 1) : n;
+  int64_t blocks = (items + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (pairs) hash_kernel<true><<<(unsigned)blocks, 256, 0, s>>>(ids, n, seed, rows, magic, rows_out);
+  else hash_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(ids, n, seed, rows, magic, rows_out);
   return cudaGetLastError();
 }
 

@@ -46,6 +46,31 @@ def test_hash_ids_bit_exact(rows):
         m.mfet_tables_destroy(h)
 
 
+@pytest.mark.parametrize("n", [1, 2, 3, 511, 513, 100_000, 100_001])
+@pytest.mark.parametrize("shift_in,shift_out", [(0, 0), (1, 0), (0, 1), (1, 1)])
+def test_hash_ids_any_length_and_alignment(n, shift_in, shift_out):
+    """The hash kernel pairs IDs up when both arrays are 16-byte aligned and falls back to single
+    IDs otherwise; odd lengths and 8-byte-aligned arrays give the same rows."""
+    m = mfet()
+    rng = np.random.default_rng(n + 10 * shift_in + 100 * shift_out)
+    rows, seed = 50_000_000, 0xC0FFEE
+    ids = rng.integers(0, 2**64 - 1, size=n, dtype=np.uint64)
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    h = m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), rows, 4, m.F32, m.LOC_DEVICE, 0, seed, 0)])
+    try:
+        buf_in = torch.zeros(n + 2, dtype=torch.int64, device="cuda")
+        buf_out = torch.full((n + 2,), -7, dtype=torch.int64, device="cuda")
+        d_ids = buf_in[shift_in:shift_in + n]
+        d_ids.copy_(torch.from_numpy(ids.view(np.int64)))
+        d_rows = buf_out[shift_out:shift_out + n]
+        m.mfet_hash_ids(h, 0, d_ids, n, d_rows, _stream())
+        assert np.array_equal(d_rows.cpu().numpy(), orc.hash_ids(ids, seed, rows))
+        out = buf_out.cpu().numpy()
+        assert (out[:shift_out] == -7).all() and (out[shift_out + n:] == -7).all()  # nothing written outside
+    finally:
+        m.mfet_tables_destroy(h)
+
+
 # ------------------------------------------------------------------ fill ----
 
 @pytest.mark.parametrize("dtype", [gi.F32, gi.F16, gi.BF16])
