@@ -424,7 +424,10 @@ __device__ __forceinline__ void pool_window_dt(const BagParams& p, const SlotDev
 
 // IDs (and weights) a thread requests before the tile's bags are ordered, so
 // that their latency overlaps the ordering.
-constexpr int kEarly = 4;
+#ifndef MFET_BAG_EARLY
+#define MFET_BAG_EARLY 8
+#endif
+constexpr int kEarly = MFET_BAG_EARLY;
 
 // Q4 = true: the build of the kernel that also decodes INT4 rows (kept apart so that the
 // common kernels stay small).
@@ -483,10 +486,13 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
     if constexpr (IND) {
       srow[pos] = (uint32_t)__ldg(ip.src + (uint32_t)id);
     } else {
-      uint64_t row = pre ? id : mod_rows(splitmix64(id ^ s.seed), s.rows, s.magic);
-      if (row >= s.rows) {
-        atomicOr(p.err, (uint32_t)MFET_DEV_ROW_RANGE);
-        row = ~0ULL;  // sentinel: no row
+      uint64_t row = mod_rows(splitmix64(id ^ s.seed), s.rows, s.magic);
+      if (pre) {  // the caller's row indices are used as they are, and checked
+        row = id;
+        if (row >= s.rows) {
+          atomicOr(p.err, (uint32_t)MFET_DEV_ROW_RANGE);
+          row = ~0ULL;  // sentinel: no row
+        }
       }
       srow[pos] = (uint32_t)row;
       if (wide) shi[pos] = (uint32_t)(row >> 32);
@@ -586,9 +592,24 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
         if (wsum) sw[pos] = ew[k];
       }
     }
-    for (int pos = tid + kEarly * 256; pos < wn; pos += 256) {
-      stage(pos, fetch_id(g0 + pos));
-      if (wsum) sw[pos] = __ldcs(p.weights + g0 + pos);
+    // the rest of a large window, again with the loads of a batch requested before any of them is used
+    for (int base = tid + kEarly * 256; base < wn; base += kEarly * 256) {
+#pragma unroll
+      for (int k = 0; k < kEarly; ++k) {
+        const int pos = base + k * 256;
+        if (pos < wn) {
+          eid[k] = fetch_id(g0 + pos);
+          if (wsum) ew[k] = __ldcs(p.weights + g0 + pos);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < kEarly; ++k) {
+        const int pos = base + k * 256;
+        if (pos < wn) {
+          stage(pos, eid[k]);
+          if (wsum) sw[pos] = ew[k];
+        }
+      }
     }
     __syncthreads();
     if (p.group_policy == 1) n_long = 0;
