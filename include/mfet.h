@@ -164,8 +164,9 @@ MFET_API int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape
  * CPU side is started as early as possible so that it runs in parallel with the rest of
  * serving and adds no latency). For a batch with exactly ONE host-table slot this runs that
  * slot's hash -> dedup -> cache probe -> fetch of the missed rows now, on the library's
- * internal stream (ordered after what `stream` holds at the call, not joined back to it),
- * into one of two result sets of the workspace. The matching mfet_embedding_bag_forward
+ * internal streams (ordered after what `stream` holds at the call, not joined back to it;
+ * the fetch has a stream of its own, so the dedup of one batch runs while the rows of the
+ * batch before it still cross PCIe), into one of two result sets of the workspace. The matching mfet_embedding_bag_forward
  * call - same ids/offsets contents, shape.flags | MFET_BATCH_PREFETCHED - then only pools,
  * and gives the same bits as a call without prefetch. At most two prefetches may be
  * outstanding; they are consumed in order. ids/offsets must stay unchanged until the

@@ -101,6 +101,11 @@ int mfet_tables_create(const mfet_table_desc_t* descs, int32_t n_tables, int32_t
   int prio_lo = 0, prio_hi = 0;
   ok = ok && cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess;
   ok = ok && cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithPriority(&h->fetch, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
+  for (int i = 0; i < 2; ++i) {
+    ok = ok && cudaEventCreateWithFlags(&h->ev_dedup[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&h->ev_fetch[i], cudaEventDisableTiming) == cudaSuccess;
+  }
   ok = ok && cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
@@ -117,6 +122,14 @@ int mfet_tables_destroy(mfet_tables_t* t) {
   if (t->side) {
     cudaStreamSynchronize(t->side);
     cudaStreamDestroy(t->side);
+  }
+  if (t->fetch) {
+    cudaStreamSynchronize(t->fetch);
+    cudaStreamDestroy(t->fetch);
+  }
+  for (int i = 0; i < 2; ++i) {
+    if (t->ev_dedup[i]) cudaEventDestroy(t->ev_dedup[i]);
+    if (t->ev_fetch[i]) cudaEventDestroy(t->ev_fetch[i]);
   }
   if (t->ev_fork) cudaEventDestroy(t->ev_fork);
   if (t->ev_join) cudaEventDestroy(t->ev_join);

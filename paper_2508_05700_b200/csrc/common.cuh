@@ -44,8 +44,12 @@ struct mfet_tables {
   std::vector<mfet::TableHost> tables;
   uint32_t* err_host = nullptr;  // pinned + mapped status word
   uint32_t* err_dev = nullptr;   // its device-visible address
-  cudaStream_t side = nullptr;   // host-table slots run here
+  cudaStream_t side = nullptr;   // host-table slots: hash + dedup + cache probe, and the pooling, run here
+  cudaStream_t fetch = nullptr;  // ... and the reads of the missed rows from host memory here, so that the
+                                 // dedup of the next batch runs while the rows of this one cross PCIe
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaEvent_t ev_dedup[2] = {nullptr, nullptr}, ev_fetch[2] = {nullptr, nullptr};  // per result set
+  int last_set = 0;              // result set of the most recent host-table batch
   void* ws = nullptr;
   uint64_t ws_bytes = 0;
   int64_t ws_max_ids = 0;
@@ -187,7 +191,7 @@ struct CacheDev {
 struct WsLayout {
   uint64_t keys_a, keys_b, idx_a, idx_b, hist, tile_counts, counters, uniq, inverse, src, miss_rows,
       staging, total;
-  uint64_t inverse2, src2, staging2;  // second result set: a prefetched batch waits here
+  uint64_t inverse2, src2, staging2, miss_rows2;  // second result set: a prefetched batch waits here
   int nblk_sort, nblk_scan;
 };
 

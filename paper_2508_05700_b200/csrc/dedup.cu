@@ -420,6 +420,7 @@ uint64_t workspace_layout(int64_t max_ids, uint64_t max_row_bytes, WsLayout* L) 
   l.inverse2 = take(n * 4);
   l.src2 = take(n * 4);
   l.staging2 = take(n * max_row_bytes);
+  l.miss_rows2 = take(n * 8);
   l.total = off;
   if (L) *L = l;
   return off;

@@ -109,22 +109,31 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
   a.n_unique = counters;
   a.src = (int32_t*)(ws + (set ? L.src2 : L.src));
   uint8_t* staging = ws + (set ? L.staging2 : L.staging);
-  a.miss_rows = (int64_t*)(ws + L.miss_rows);
-  a.n_miss = counters + 1;
+  a.miss_rows = (int64_t*)(ws + (set ? L.miss_rows2 : L.miss_rows));
+  a.n_miss = counters + 1 + set;
   a.err = t->err_dev;
   const bool prof = t->profile != 0 && stage == 3;
   const uint32_t chunks = (uint32_t)(tb.row_bytes / 16);
   if (prof) cudaEventRecord(t->prof_ev[0], side);
   if (stage & 1) {
+    // hash + dedup + probe on the side stream; the reads of the missed rows on the fetch stream, which
+    // the next batch's dedup does not wait for (it writes the other result set)
     if (launch_dedup(a, &t->launches, side) != cudaSuccess) return MFET_ERR_CUDA;
     if (prof) cudaEventRecord(t->prof_ev[1], side);
-    if (launch_fetch(tb.dev_ptr, tb.stride, chunks, a.miss_rows, a.n_miss, 0, staging, side) != cudaSuccess)
+    if (cudaEventRecord(t->ev_dedup[set], side) != cudaSuccess) return MFET_ERR_CUDA;
+    if (cudaStreamWaitEvent(t->fetch, t->ev_dedup[set], 0) != cudaSuccess) return MFET_ERR_CUDA;
+    if (launch_fetch(tb.dev_ptr, tb.stride, chunks, a.miss_rows, a.n_miss, 0, staging, t->fetch) != cudaSuccess)
       return MFET_ERR_CUDA;
     t->launches += 1;
-    if (prof) cudaEventRecord(t->prof_ev[2], side);
+    if (prof) cudaEventRecord(t->prof_ev[2], t->fetch);
+    if (cudaEventRecord(t->ev_fetch[set], t->fetch) != cudaSuccess) return MFET_ERR_CUDA;
+    t->last_set = set;
   }
   if (!(stage & 2)) return MFET_OK;
 
+  // the pooling follows on the side stream once the set's rows have arrived; a later dedup into the
+  // same set is behind it in that stream
+  if (cudaStreamWaitEvent(side, t->ev_fetch[set], 0) != cudaSuccess) return MFET_ERR_CUDA;
   IndirectParams ip{a.inverse, a.src, tb.cache.data, staging, tb.row_bytes, t->ws_max_ids};
   BagParams p = base;
   p.flags &= ~1u;  // the indirect path never hashes
@@ -209,13 +218,13 @@ int mfet_host_path_counts(mfet_tables_t* t, int64_t* n_unique, int64_t* n_miss) 
   int prev = 0;
   if (cudaGetDevice(&prev) != cudaSuccess) return MFET_ERR_CUDA;
   if (prev != t->device && cudaSetDevice(t->device) != cudaSuccess) return MFET_ERR_CUDA;
-  int64_t c[2] = {0, 0};
-  bool ok = cudaStreamSynchronize(t->side) == cudaSuccess &&
+  int64_t c[3] = {0, 0, 0};  // n_unique, n_miss of result set 0, of result set 1
+  bool ok = cudaStreamSynchronize(t->side) == cudaSuccess && cudaStreamSynchronize(t->fetch) == cudaSuccess &&
             cudaMemcpy(c, static_cast<uint8_t*>(t->ws) + L.counters, sizeof(c), cudaMemcpyDeviceToHost) == cudaSuccess;
   if (prev != t->device) cudaSetDevice(prev);
   if (!ok) return MFET_ERR_CUDA;
   *n_unique = c[0];
-  *n_miss = c[1];
+  *n_miss = c[1 + (t->last_set & 1)];
   return MFET_OK;
 }
 
