@@ -703,6 +703,41 @@ def test_prefetched_batches_give_the_same_bits_as_the_serial_path():
             assert e.status == m.ERR_INVALID_ARG
 
 
+def test_early_fetch_pipeline_in_steady_state():
+    """Every step announces its successor (prefetch of batch j+1, then the pooling of batch j), for many
+    steps over rotating batches and without a synchronisation in between: the dedup of one batch runs
+    while the rows of another are fetched and a third is pooled, and every result has the serial path's bits."""
+    m = mfet()
+    w = gi.make_workload(5, rows_scale=0.001, batch_scale=0.125)
+    bs = [gi.make_batch(w, j) for j in range(3)]
+    cap = max(int(b.offsets[w.batch] - b.offsets[0]) for b in bs) + 1024
+    with DeviceTables(w.tables) as dt:
+        dt.set_workspace(cap)
+        dt.build_cache(0, _hot_rows(dt, w, 0, 0, int(w.tables[0].rows * 0.02), w.tables[0].rows))
+        serial = [workload_forward(dt, w, b) for b in bs]
+        d_ids = [torch.from_numpy(b.ids.view(np.int64)).cuda() for b in bs]
+        d_off = [torch.from_numpy(b.offsets).cuda() for b in bs]
+        steps = 10
+        outs = [torch.full((w.batch, w.out_dim), float("nan"), device="cuda") for _ in range(steps)]
+        plain, keep = m.make_shape(w.batch, w.n_features, w.slot_feature)
+        pre, keep2 = m.make_shape(w.batch, w.n_features, w.slot_feature)
+        pre.flags |= m.BATCH_PREFETCHED
+        s = _stream()
+        m.mfet_host_prefetch(dt.h, plain, d_ids[0], d_off[0], w.table_ids, s)
+        for j in range(steps):
+            k, kn = j % 3, (j + 1) % 3
+            if j + 1 < steps:
+                m.mfet_host_prefetch(dt.h, plain, d_ids[kn], d_off[kn], w.table_ids, s)
+            m.mfet_embedding_bag_forward(dt.h, pre, d_ids[k], d_off[k], None, w.table_ids, w.pooling, outs[j], s)
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(dt.h) == 0
+        for j in range(steps):
+            assert np.array_equal(outs[j].cpu().numpy(), serial[j % 3]), j
+        n_unique, n_miss = m.mfet_host_path_counts(dt.h)
+        assert 0 < n_miss <= n_unique <= cap
+        assert np.array_equal(workload_forward(dt, w, bs[1]), serial[1])  # and the serial path afterwards
+
+
 def test_version_tag_is_echoed_unchanged():
     """Paper, Algorithm 2: embeddings are returned together with the version of the tables."""
     m = mfet()
