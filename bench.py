@@ -321,6 +321,10 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
 
     dev = torch.cuda.current_device()
     eng = LookupEngine(w, device=dev)
+    if not args.no_overlap_launches:
+        # the batches are resident before the timed region: a step's kernel may hash its IDs while the
+        # step before it finishes (it waits for that kernel before it writes the output)
+        m.mfet_set_option(eng.h, m.OPT_OVERLAP_LAUNCHES, 1)
     if args.tile:
         m.mfet_set_option(eng.h, m.OPT_TILE, args.tile)
     if args.stage_ids:
@@ -409,22 +413,35 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
     assert m.mfet_query_status(eng.h) == 0, "device error bits set during the timed region"
 
     # ---- the pooling kernel alone: all HBM-resident slots, one launch per step ----
+    # timed as in the timed region (launches may overlap by their start-up phase) and with every launch
+    # waiting for the one before it ("serialized": the duration of a launch by itself)
     dev_slots = [s for s in range(w.n_slots) if w.tables[int(w.table_ids[s])].location == gi.LOC_DEVICE]
-    if len(dev_slots) == w.n_slots:
-        kern_ms = local_ms / args.steps
-    else:
+    all_dev = len(dev_slots) == w.n_slots
+    if not all_dev:
         sub_shape, keep = m.make_shape(w.batch, w.n_features, w.slot_feature[dev_slots])
         sub_out = torch.empty(w.batch, sum(w.tables[int(w.table_ids[s])].dim for s in dev_slots), device="cuda")
+
+    def kernel_alone_ms():
         k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         for rep in range(2):
             k0.record(stream)
             for j in range(args.steps):
                 k = j % n_rot
-                eng.forward(d_ids[k], d_off[k], d_w[k], sub_out, table_ids=w.table_ids[dev_slots],
-                            pooling=w.pooling[dev_slots], shape=sub_shape)
+                if all_dev:
+                    eng.forward(d_ids[k], d_off[k], d_w[k], out)
+                else:
+                    eng.forward(d_ids[k], d_off[k], d_w[k], sub_out, table_ids=w.table_ids[dev_slots],
+                                pooling=w.pooling[dev_slots], shape=sub_shape)
             k1.record(stream)
             torch.cuda.synchronize()
-        kern_ms = k0.elapsed_time(k1) / args.steps
+        return k0.elapsed_time(k1) / args.steps
+
+    kern_ms = local_ms / args.steps if all_dev else kernel_alone_ms()
+    kern_ms_serialized = kern_ms
+    if not args.no_overlap_launches:
+        m.mfet_set_option(eng.h, m.OPT_OVERLAP_LAUNCHES, 0)
+        kern_ms_serialized = kernel_alone_ms()
+        m.mfet_set_option(eng.h, m.OPT_OVERLAP_LAUNCHES, 1)
     alg = float(np.mean([algorithmic_bytes(w, batches[j % n_rot], dev_slots) for j in range(min(args.steps, n_rot))]))
 
     # ---- host-table path alone (PCIe roofline): stage times from the library's events ----
@@ -556,13 +573,18 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
                    "table_bytes": int(sum(t.rows * gi_row_bytes(t) for t in w.tables)),
                    "rows_scale": args.rows_scale, "cached_rows": cached_rows,
                    "l2": "no flush: tables are far larger than L2 and %d distinct batches rotate" % n_rot,
+                   "launch_overlap": not args.no_overlap_launches,
                    "parallelism": "replicas x%d" % world},
         "e2e": {"value": units / (e2e_ms_all * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": recorded_traffic(wl_key), "peak_kind": peak_kind + " copy bandwidth",
                      "kernel": "bag_kernel (all HBM-resident slots, one launch)",
-                     "algorithmic_bytes_per_launch": alg, "kernel_ms": kern_ms},
+                     "algorithmic_bytes_per_launch": alg, "kernel_ms": kern_ms,
+                     "serialized": {"kernel_ms": kern_ms_serialized,
+                                    "achieved": alg / (kern_ms_serialized * 1e-3) / 1e9,
+                                    "frac": alg / (kern_ms_serialized * 1e-3) / 1e9 / peak,
+                                    "note": "every launch waits for the one before it (no programmatic dependent launch)"}},
         "roofline_host_path": host_path,
         "stages_alone": alone,
         "cpu_baseline": base,
@@ -618,6 +640,8 @@ def main():
     ap.add_argument("--batches", type=int, default=8, help="distinct batches rotated through")
     ap.add_argument("--load-seconds", type=float, default=1.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap-launches", action="store_true",
+                    help="every pooling kernel starts only when the kernel before it on the stream has finished")
     ap.add_argument("--serial-host-path", action="store_true",
                     help="hybrid workload: no early fetch of the next batch's host-table rows")
     ap.add_argument("--device-slots-only", action="store_true",

@@ -48,7 +48,8 @@ enum { MFET_POOL_SUM = 0, MFET_POOL_MEAN = 1, MFET_POOL_WSUM = 2 };
 enum { MFET_LOC_DEVICE = 0, MFET_LOC_HOST = 1 };
 enum { MFET_VAL_NORMAL = 0, MFET_VAL_GRID = 1 };
 enum { MFET_BATCH_IDS_ARE_ROWS = 1, MFET_BATCH_PREFETCHED = 2 }; /* mfet_batch_shape_t.flags */
-enum { MFET_OPT_GROUP_POLICY = 1, MFET_OPT_TILE = 2, MFET_OPT_PROFILE = 3, MFET_OPT_STAGE_IDS = 4 };
+enum { MFET_OPT_GROUP_POLICY = 1, MFET_OPT_TILE = 2, MFET_OPT_PROFILE = 3, MFET_OPT_STAGE_IDS = 4,
+       MFET_OPT_OVERLAP_LAUNCHES = 5 };
 
 enum {
   MFET_OK = 0,
@@ -313,7 +314,14 @@ MFET_API int mfet_query_status(mfet_tables_t* t, uint32_t* device_error_bits /*h
  * how many IDs of a tile the pooling kernel hashes into shared memory at a time:
  * 0 = default (4096), or 32 .. 8192; a tile with more
  * IDs is pooled in several passes and a bag cut by a pass boundary continues from
- * its partial sum (same result up to the order of fp32 additions). MFET_OPT_PROFILE:
+ * its partial sum (same result up to the order of fp32 additions).
+ * MFET_OPT_OVERLAP_LAUNCHES: 1 = the pooling kernel of a forward call may begin while the
+ * kernel launched before it on the same stream is still running (programmatic dependent
+ * launch): it reads its offsets, IDs and weights and hashes them, and waits for that kernel
+ * to complete before it writes `out` or reads it. Only for callers whose ids / offsets /
+ * weights are NOT written by the kernel that precedes the call on the stream (copies that
+ * precede it are waited for as usual); back-to-back forward calls then overlap by the
+ * start-up phase of a launch. Default 0. MFET_OPT_PROFILE:
  * 1 = record CUDA events around the stages of the host-table path of every forward
  * call (read them with mfet_profile_read). */
 MFET_API int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value);

@@ -248,6 +248,10 @@ int mfet_set_option(mfet_tables_t* t, int32_t option, int64_t value) {
       if (value != 0 && (value < 8 || value > kMaxTile)) return MFET_ERR_INVALID_ARG;
       t->tile = (int32_t)value;
       return MFET_OK;
+    case MFET_OPT_OVERLAP_LAUNCHES:
+      if (value != 0 && value != 1) return MFET_ERR_INVALID_ARG;
+      t->overlap = (int32_t)value;
+      return MFET_OK;
     case MFET_OPT_STAGE_IDS:
       if (value != 0 && (value < 32 || value > kStageMax)) return MFET_ERR_INVALID_ARG;
       t->stage_cap = (int32_t)value;
@@ -394,6 +398,7 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
   p.batch = B;
   p.flags = (uint32_t)(shape->flags & 1);
   if (aligned16(out) && out_ld % 4 == 0) p.flags |= 2u;
+  if (t->overlap) p.flags |= 16u;
   p.group_policy = t->group_policy;
   // samples per block and staging capacity: the caller's options, else chosen at launch (0)
   p.tile = t->tile;

@@ -443,6 +443,11 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   __shared__ int scnt[kSortWarps][kClasses + 1];
   __shared__ int snext;
   const int tid = threadIdx.x;
+  // Launched with programmatic stream serialisation (flag bit 4), the blocks of the NEXT launch on the
+  // stream may start as soon as every block of this one has got here; they read and hash their own
+  // inputs, then wait below until this launch is complete. Without that launch attribute both
+  // instructions do nothing.
+  asm volatile("griddepcontrol.launch_dependents;");
   const int slot = blockIdx.x / p.tiles_per_slot;
   const int tile = blockIdx.x - slot * p.tiles_per_slot;
   const SlotDev& s = p.slot[slot];
@@ -612,6 +617,8 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
       }
     }
     __syncthreads();
+    // nothing of the stream's earlier kernel is touched before this point, nothing is written before it
+    if (w0 == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (p.group_policy == 1) n_long = 0;
     if (p.group_policy == 2) n_long = nbw;
 
@@ -786,6 +793,22 @@ static void prepare(K kernel, int which, size_t smem) {
   configured[which][dev].store(want, std::memory_order_relaxed);
 }
 
+// Launch with or without permission to start before the stream's previous kernel has finished.
+template <typename K, typename... Args>
+static cudaError_t launch(K kernel, int64_t blocks, size_t smem, cudaStream_t s, bool overlap, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)blocks);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = overlap ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 cudaError_t launch_bag_indirect(const BagParams& p_, const IndirectParams& ip, cudaStream_t s) {
   BagParams p = p_;
   if (p.n_slots == 0 || p.batch <= 0) return cudaSuccess;
@@ -793,12 +816,10 @@ cudaError_t launch_bag_indirect(const BagParams& p_, const IndirectParams& ip, c
   const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
   if (any_int4(p)) {
     prepare(bag_indirect_q4_kernel, 0, smem);
-    bag_indirect_q4_kernel<<<(unsigned)blocks, 256, smem, s>>>(p, ip);
-  } else {
-    prepare(bag_indirect_kernel, 1, smem);
-    bag_indirect_kernel<<<(unsigned)blocks, 256, smem, s>>>(p, ip);
+    return launch(bag_indirect_q4_kernel, blocks, smem, s, false, p, ip);
   }
-  return cudaGetLastError();
+  prepare(bag_indirect_kernel, 1, smem);
+  return launch(bag_indirect_kernel, blocks, smem, s, false, p, ip);
 }
 
 cudaError_t launch_bag(const BagParams& p_, cudaStream_t s) {
@@ -806,14 +827,13 @@ cudaError_t launch_bag(const BagParams& p_, cudaStream_t s) {
   if (p.n_slots == 0 || p.batch <= 0) return cudaSuccess;
   const size_t smem = stage_bytes(p, false);
   const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
+  const bool overlap = (p.flags & 16u) != 0;
   if (any_int4(p)) {
     prepare(bag_q4_kernel, 2, smem);
-    bag_q4_kernel<<<(unsigned)blocks, 256, smem, s>>>(p);
-  } else {
-    prepare(bag_kernel, 3, smem);
-    bag_kernel<<<(unsigned)blocks, 256, smem, s>>>(p);
+    return launch(bag_q4_kernel, blocks, smem, s, overlap, p);
   }
-  return cudaGetLastError();
+  prepare(bag_kernel, 3, smem);
+  return launch(bag_kernel, blocks, smem, s, overlap, p);
 }
 
 }  // namespace mfet

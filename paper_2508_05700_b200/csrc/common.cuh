@@ -59,6 +59,7 @@ struct mfet_tables {
   uint64_t prefetched = 0, consumed = 0;  // batches handed to mfet_host_prefetch / pooled from a prefetch
   int32_t tile = 0;  // bags per block; 0 = chosen from the batch size
   int32_t stage_cap = 0;  // IDs staged per window of the pooling kernel; 0 = default
+  int32_t overlap = 0;    // 1: pooling launches may begin while the stream's previous kernel still runs
   int32_t profile = 0;             // 1: time the stages of the host-table path with events
   cudaEvent_t prof_ev[4] = {nullptr, nullptr, nullptr, nullptr};
   bool prof_valid = false;
@@ -107,7 +108,8 @@ struct BagParams {
   int32_t tiles_per_slot;
   int32_t tile;          // bags per block, <= kMaxTile
   uint32_t flags;        // bit0: ids are rows; bit1: out allows 16-byte vector stores;
-                         // set at launch: bit2 weights are staged, bit3 upper row-index halves are staged
+                         // set at launch: bit2 weights are staged, bit3 upper row-index halves are staged;
+                         // bit4: the launch may begin before the stream's previous kernel has finished
   int32_t group_policy;  // 0 auto, 1 one row-group per bag, 2 one warp per bag
   int32_t stage_cap;     // IDs staged per window, 32 .. kStageMax (0: default)
   SlotDev slot[kMaxSlotsPerLaunch];

@@ -25,6 +25,7 @@ OPT_GROUP_POLICY = 1
 OPT_TILE = 2
 OPT_PROFILE = 3
 OPT_STAGE_IDS = 4
+OPT_OVERLAP_LAUNCHES = 5
 OK = 0
 ERR_INVALID_ARG, ERR_NOT_REGISTERED, ERR_ALIGNMENT, ERR_UNSUPPORTED_DIM = -1, -2, -3, -4
 ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7

@@ -286,6 +286,41 @@ def test_stage_option_range():
         mt.close()
 
 
+def test_overlapping_launches_give_the_same_bits():
+    """MFET_OPT_OVERLAP_LAUNCHES: back-to-back forward calls on one stream, into the same output buffer
+    and into different ones, with a consumer kernel between them; every result has the bits of the
+    serialised launches and matches the oracle."""
+    w = gi.make_workload(3, rows_scale=1e-3, batch_scale=1 / 8)
+    bs = [gi.make_batch(w, j) for j in range(4)]
+    with DeviceTables(w.tables) as dt:
+        m = dt.m
+        serial = [workload_forward(dt, w, b) for b in bs]
+        assert_close(serial[0], workload_oracle(dt, w, bs[0]))
+        m.mfet_set_option(dt.h, m.OPT_OVERLAP_LAUNCHES, 1)
+        d = [(torch.from_numpy(b.ids.view(np.int64)).cuda(), torch.from_numpy(b.offsets).cuda(),
+              torch.from_numpy(b.weights).cuda()) for b in bs]
+        shape, keep = m.make_shape(w.batch, w.n_features, w.slot_feature)
+        torch.cuda.synchronize()
+        s = _stream()
+        out = torch.empty(w.batch, w.out_dim, dtype=torch.float32, device="cuda")
+        copies = []
+        for rep in range(3):
+            for j in range(4):
+                m.mfet_embedding_bag_forward(dt.h, shape, d[j][0], d[j][1], d[j][2], w.table_ids, w.pooling, out, s)
+                copies.append((j, out.clone()))  # a kernel that reads the result, between two forward calls
+        outs = [torch.empty_like(out) for _ in range(4)]
+        for j in range(4):  # and directly back to back into different buffers
+            m.mfet_embedding_bag_forward(dt.h, shape, d[j][0], d[j][1], d[j][2], w.table_ids, w.pooling, outs[j], s)
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(dt.h) == 0
+        for j, c in copies:
+            assert np.array_equal(c.cpu().numpy(), serial[j]), j
+        for j in range(4):
+            assert np.array_equal(outs[j].cpu().numpy(), serial[j]), j
+        with pytest.raises(m.MfetError):
+            m.mfet_set_option(dt.h, m.OPT_OVERLAP_LAUNCHES, 2)
+
+
 def test_single_row_table_and_prehashed_rows():
     rng = np.random.default_rng(3)
     tab = rng.standard_normal((1, 32)).astype(np.float32)
