@@ -47,9 +47,25 @@ def test_full_size_sampled_parity(config):
         torch.cuda.synchronize()
         assert m.mfet_query_status(eng.h) == 0
         first = out.clone()
-        eng.forward(d_ids, d_off, d_w, out)
+        # as the benchmark launches it: back to back, a launch may begin while the one before it finishes
+        m.mfet_set_option(eng.h, m.OPT_OVERLAP_LAUNCHES, 1)
+        for _ in range(3):
+            eng.forward(d_ids, d_off, d_w, out)
         torch.cuda.synchronize()
         assert torch.equal(first, out)                       # fixed summation order
+        if eng.host_table_ids():
+            # ... and with the early fetch of the next batch's host-table rows
+            pre, _keep = m.make_shape(w.batch, w.n_features, w.slot_feature)
+            pre.flags |= m.BATCH_PREFETCHED
+            out.fill_(float("nan"))
+            m.mfet_host_prefetch(eng.h, eng.shape, d_ids, d_off, w.table_ids, eng.stream)
+            for k in range(3):
+                if k < 2:
+                    m.mfet_host_prefetch(eng.h, eng.shape, d_ids, d_off, w.table_ids, eng.stream)
+                m.mfet_embedding_bag_forward(eng.h, pre, d_ids, d_off, d_w, w.table_ids, w.pooling, out, eng.stream)
+            torch.cuda.synchronize()
+            assert torch.equal(first, out)
+        assert m.mfet_query_status(eng.h) == 0
         assert bool(torch.isfinite(out).all())
         # empty bags give exact zeros in their slot's columns (all samples, on the GPU)
         lens = torch.from_numpy(np.diff(b.offsets).reshape(w.n_features, w.batch)).cuda()
