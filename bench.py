@@ -575,7 +575,10 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
                    "l2": "no flush: tables are far larger than L2 and %d distinct batches rotate" % n_rot,
                    "launch_overlap": not args.no_overlap_launches,
                    "parallelism": "replicas x%d" % world},
-        "e2e": {"value": units / (e2e_ms_all * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "e2e": {"value": units / (e2e_ms_all * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                # the two directions of the link run at the same time; the busier one bounds the step
+                "link_gbps": max(h2d, d2h) * args.steps / (e2e_ms_all * 1e-3) / 1e9,  # per GPU
+                "link_direction": "d2h" if d2h >= h2d else "h2d"},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": recorded_traffic(wl_key), "peak_kind": peak_kind + " copy bandwidth",
