@@ -27,8 +27,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     procs = []
     for s in srcs:
         o = os.path.join(CSRC, os.path.basename(s)[:-3] + ".o")
-        extra = os.environ.get("MFET_NVCC_EXTRA", "").split()  # e.g. -DMFET_BAG_U=8 for a tuning sweep
-        cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
         procs.append((cmd, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(o)
     for cmd, p in procs:

@@ -1,6 +1,7 @@
 // C-ABI boundary: argument checking, descriptor bookkeeping and launch
 // orchestration. No arithmetic of the lookup path happens on the host.
 #include <algorithm>
+#include <atomic>
 #include <cstring>
 #include <new>
 
@@ -27,6 +28,25 @@ struct DeviceGuard {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
+
+namespace mfet {
+
+int sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  int sms = cached[dev].load(std::memory_order_relaxed);
+  if (sms == 0) {
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+      cudaGetLastError();
+      return 148;  // not cached: asked again next time
+    }
+    cached[dev].store(sms, std::memory_order_relaxed);
+  }
+  return sms;
+}
+
+}  // namespace mfet
 
 extern "C" {
 

@@ -73,7 +73,7 @@ cudaError_t launch_backward(const uint32_t* sorted_pos, const int32_t* seg_start
                             const int64_t* offsets_f, int32_t batch, const float* weights, int32_t pooling,
                             const float* grad_out, int64_t out_ld, uint32_t col, uint32_t dim, float* grad_vals,
                             cudaStream_t s) {
-  backward_rows_kernel<<<148 * 8, 256, 0, s>>>(sorted_pos, seg_start, n_unique, ns, offsets_f, batch, weights, pooling,
+  backward_rows_kernel<<<sm_count() * 8, 256, 0, s>>>(sorted_pos, seg_start, n_unique, ns, offsets_f, batch, weights, pooling,
                                                grad_out, out_ld, col, dim, grad_vals);
   return cudaGetLastError();
 }

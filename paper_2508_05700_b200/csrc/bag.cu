@@ -35,25 +35,14 @@
 
 #include "common.cuh"
 
-// Tunables (overridable at build time for sweeps): row loads kept in flight per
-// lane, the length from which a bag gets a whole warp and the minimum number of
-// resident blocks per SM (caps registers).
-#ifndef MFET_BAG_U
-#define MFET_BAG_U 8
-#endif
-#ifndef MFET_BAG_LONG
-#define MFET_BAG_LONG 64
-#endif
-#ifndef MFET_BAG_MINB
-#define MFET_BAG_MINB 4
-#endif
-
 namespace mfet {
 
 namespace {
 
 constexpr unsigned kFull = 0xFFFFFFFFu;
-constexpr int kLongBag = MFET_BAG_LONG;  // bags at least this long get a whole warp
+constexpr int kLongBag = 64;      // bags at least this long get a whole warp (32: measured slower)
+constexpr int kGatherLoads = 8;  // row loads that a lane keeps in flight (4 with 48 registers: slower)
+constexpr int kMinBlocks = 4;    // resident blocks per SM that the register budget allows (3, 5: slower)
 // the ordering of the shorter bags has one lane per length class: classes of kClassW lengths
 constexpr int kClassW = (kLongBag + 31) / 32;
 constexpr int kClasses = (kLongBag + kClassW - 1) / kClassW;  // <= 32; class kClasses = long bags
@@ -255,7 +244,7 @@ __device__ __forceinline__ void run_steps(const uint32_t* srow, const uint32_t* 
 template <int DT, int GG, bool IND, bool WS>
 __device__ __forceinline__ int run_common(const uint32_t* srow, const float* sw, const RowAddr<IND>& ra,
                                           int min_steps, unsigned long long* acc) {
-  constexpr int U = MFET_BAG_U;
+  constexpr int U = kGatherLoads;
   int t = 0;
   for (; t + U <= min_steps; t += U)
     run_steps<DT, GG, IND, U, false, WS>(srow + t * GG, nullptr, sw + t * GG, ra, WS, 0, true, acc);
@@ -424,10 +413,7 @@ __device__ __forceinline__ void pool_window_dt(const BagParams& p, const SlotDev
 
 // IDs (and weights) a thread requests before the tile's bags are ordered, so
 // that their latency overlaps the ordering.
-#ifndef MFET_BAG_EARLY
-#define MFET_BAG_EARLY 8
-#endif
-constexpr int kEarly = MFET_BAG_EARLY;
+constexpr int kEarly = 8;
 
 // Q4 = true: the build of the kernel that also decodes INT4 rows (kept apart so that the
 // common kernels stay small).
@@ -646,22 +632,22 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   }
 }
 
-__global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_kernel(const __grid_constant__ BagParams p) {
+__global__ void __launch_bounds__(256, kMinBlocks) bag_kernel(const __grid_constant__ BagParams p) {
   const IndirectParams none{};
   bag_body<false, false>(p, none);
 }
 
-__global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_q4_kernel(const __grid_constant__ BagParams p) {
+__global__ void __launch_bounds__(256, kMinBlocks) bag_q4_kernel(const __grid_constant__ BagParams p) {
   const IndirectParams none{};
   bag_body<false, true>(p, none);
 }
 
-__global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_indirect_kernel(const __grid_constant__ BagParams p,
+__global__ void __launch_bounds__(256, kMinBlocks) bag_indirect_kernel(const __grid_constant__ BagParams p,
                                                            const __grid_constant__ IndirectParams ip) {
   bag_body<true, false>(p, ip);
 }
 
-__global__ void __launch_bounds__(256, MFET_BAG_MINB) bag_indirect_q4_kernel(const __grid_constant__ BagParams p,
+__global__ void __launch_bounds__(256, kMinBlocks) bag_indirect_q4_kernel(const __grid_constant__ BagParams p,
                                                               const __grid_constant__ IndirectParams ip) {
   bag_body<true, true>(p, ip);
 }
@@ -693,13 +679,7 @@ static int choose_tile(const BagParams& p) {
   static std::vector<Entry> memo;
   int dev = 0;
   cudaGetDevice(&dev);
-  static std::atomic<int> sm_count[64];
-  int sms = dev >= 0 && dev < 64 ? sm_count[dev].load(std::memory_order_relaxed) : 0;
-  if (sms == 0) {
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-    if (dev >= 0 && dev < 64) sm_count[dev].store(sms, std::memory_order_relaxed);
-  }
-  const int slots = sms * MFET_BAG_MINB;
+  const int slots = sm_count() * kMinBlocks;
   if ((int64_t)p.n_slots * ((p.batch + kMaxTile - 1) / kMaxTile) >= 6LL * slots) return kMaxTile;
   Entry key{};
   key.dev = dev;
@@ -773,24 +753,30 @@ static size_t stage_bytes(BagParams& p, bool indirect) {
 }
 
 // Shared-memory set-up of a kernel for a launch with `smem` dynamic bytes, redone only when
-// that size changes (per kernel and device): the opt-in above 48 KB, and a carve-out of just
-// what the resident blocks need, so that the rest of the SM's array stays L1 for the rows.
+// that size changes (per kernel and device): the opt-in that a block needs for more than 48 KB
+// of shared memory (static and dynamic together), and a carve-out of just what the resident
+// blocks need, so that the rest of the SM's array stays L1 for the rows.
 template <typename K>
-static void prepare(K kernel, int which, size_t smem) {
+static cudaError_t prepare(K kernel, int which, size_t smem) {
   static std::atomic<long long> configured[4][64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
   const long long want = (long long)smem + 1;
-  if (configured[which][dev].load(std::memory_order_relaxed) == want) return;
-  if (smem > 48 * 1024) cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStageMax * 12);
+  if (configured[which][dev].load(std::memory_order_relaxed) == want) return cudaSuccess;
   cudaFuncAttributes fa{};
-  if (cudaFuncGetAttributes(&fa, kernel) != cudaSuccess) fa.sharedSizeBytes = 4096;
+  cudaError_t e = cudaFuncGetAttributes(&fa, kernel);
+  if (e != cudaSuccess) return e;
+  if (smem + fa.sharedSizeBytes > 48 * 1024) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStageMax * 12);
+    if (e != cudaSuccess) return e;
+  }
   const size_t per_block = smem + fa.sharedSizeBytes + 1024;  // dynamic + static + the system's share
-  size_t pct = (MFET_BAG_MINB * per_block * 100 + 228 * 1024 - 1) / (228 * 1024);
+  size_t pct = (kMinBlocks * per_block * 100 + 228 * 1024 - 1) / (228 * 1024);
   if (pct > 100) pct = 100;
-  cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)pct);
-  cudaGetLastError();
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, (int)pct);
+  if (e != cudaSuccess) return e;
   configured[which][dev].store(want, std::memory_order_relaxed);
+  return cudaSuccess;
 }
 
 // Launch with or without permission to start before the stream's previous kernel has finished.
@@ -814,11 +800,12 @@ cudaError_t launch_bag_indirect(const BagParams& p_, const IndirectParams& ip, c
   if (p.n_slots == 0 || p.batch <= 0) return cudaSuccess;
   const size_t smem = stage_bytes(p, true);
   const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
+  cudaError_t e;
   if (any_int4(p)) {
-    prepare(bag_indirect_q4_kernel, 0, smem);
+    if ((e = prepare(bag_indirect_q4_kernel, 0, smem)) != cudaSuccess) return e;
     return launch(bag_indirect_q4_kernel, blocks, smem, s, false, p, ip);
   }
-  prepare(bag_indirect_kernel, 1, smem);
+  if ((e = prepare(bag_indirect_kernel, 1, smem)) != cudaSuccess) return e;
   return launch(bag_indirect_kernel, blocks, smem, s, false, p, ip);
 }
 
@@ -828,11 +815,12 @@ cudaError_t launch_bag(const BagParams& p_, cudaStream_t s) {
   const size_t smem = stage_bytes(p, false);
   const int64_t blocks = (int64_t)p.n_slots * p.tiles_per_slot;
   const bool overlap = (p.flags & 16u) != 0;
+  cudaError_t e;
   if (any_int4(p)) {
-    prepare(bag_q4_kernel, 2, smem);
+    if ((e = prepare(bag_q4_kernel, 2, smem)) != cudaSuccess) return e;
     return launch(bag_q4_kernel, blocks, smem, s, overlap, p);
   }
-  prepare(bag_kernel, 3, smem);
+  if ((e = prepare(bag_kernel, 3, smem)) != cudaSuccess) return e;
   return launch(bag_kernel, blocks, smem, s, overlap, p);
 }
 

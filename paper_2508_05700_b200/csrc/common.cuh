@@ -139,23 +139,16 @@ __device__ __forceinline__ uint64_t mod_rows(uint64_t h, uint64_t d, uint64_t ma
 
 inline uint64_t host_magic(uint64_t rows) { return 0xFFFFFFFFFFFFFFFFULL / rows; }
 
+// Number of SMs of the current device (asked once per device; grids are sized by it).
+int sm_count();
+
 // 16-byte row load through the read-only path. Rows may allocate in L1: with Zipf-distributed
 // IDs an SM re-reads the head rows of a table hundreds of times per batch, and serving those
-// from L1 measured 2-8 % faster than keeping rows out of it.
-#ifndef MFET_ROW_LD
-#define MFET_ROW_LD 1  // 0 no L1 allocation, 1 default, 2 evict-last, 3 evict-first (measured: 1 is best)
-#endif
+// from L1 measured 2-8 % faster than keeping rows out of it (no allocation, evict-first and
+// evict-last hints were all slower).
 __device__ __forceinline__ uint4 ld_row16(const void* p) {
   uint4 v;
-#if MFET_ROW_LD == 0
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-#elif MFET_ROW_LD == 1
   asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
-#elif MFET_ROW_LD == 2
-  asm volatile("ld.global.nc.L1::evict_last.v4.u32 {%0,%1,%2,%3}, [%4];"
-#else
-  asm volatile("ld.global.nc.L1::evict_first.v4.u32 {%0,%1,%2,%3}, [%4];"
-#endif
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                : "l"(p));
   return v;

@@ -52,7 +52,7 @@ cudaError_t launch_hash(const uint64_t* ids, int64_t n, uint64_t seed, uint64_t 
   const bool pairs = n >= 2 && ((reinterpret_cast<uintptr_t>(ids) | reinterpret_cast<uintptr_t>(rows_out)) & 15u) == 0;
   const int64_t items = pairs ? (n >> 1) : n;
   int64_t blocks = (items + 255) / 256;
-  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks > sm_count() * 8) blocks = sm_count() * 8;
   if (pairs) hash_kernel<true><<<(unsigned)blocks, 256, 0, s>>>(ids, n, seed, rows, magic, rows_out);
   else hash_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(ids, n, seed, rows, magic, rows_out);
   return cudaGetLastError();
@@ -156,7 +156,7 @@ cudaError_t launch_fill(void* data, uint64_t row0, uint64_t n_rows, uint32_t dim
   const uint32_t chunks = (uint32_t)(mfet_row_bytes(dim, dtype) / 16);
   uint64_t total = n_rows * chunks;
   uint64_t blocks = (total + 255) / 256;
-  if (blocks > 148ull * 32) blocks = 148ull * 32;
+  if (blocks > (uint64_t)sm_count() * 32) blocks = (uint64_t)sm_count() * 32;
   fill_kernel<<<(unsigned)blocks, 256, 0, s>>>((uint8_t*)data, row0, n_rows, dim, dtype, stride, key,
                                                mode, chunks);
   return cudaGetLastError();

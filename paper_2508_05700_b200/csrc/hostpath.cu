@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(256) cache_index_kernel(const int64_t* __restr
 
 cudaError_t launch_fetch(const uint8_t* table, uint64_t stride, uint32_t chunks, const int64_t* rows_list,
                          const int64_t* n_ptr, int64_t n_imm, uint8_t* dst, cudaStream_t s) {
-  fetch_rows_kernel<<<148 * 4, 256, 0, s>>>(table, stride, chunks, rows_list, n_ptr, n_imm, dst);
+  fetch_rows_kernel<<<sm_count() * 4, 256, 0, s>>>(table, stride, chunks, rows_list, n_ptr, n_imm, dst);
   return cudaGetLastError();
 }
 

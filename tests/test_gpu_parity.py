@@ -286,6 +286,48 @@ def test_stage_option_range():
         mt.close()
 
 
+@pytest.mark.parametrize("stage", [4095, 5755, 6000, 6144, 8192])
+def test_large_staging_capacities_launch(stage):
+    """Staging capacities whose shared memory per block lies just under, around and above 48 KB
+    (static and dynamic together; a weighted slot stages 8 bytes per ID): the launch is accepted
+    and matches the oracle."""
+    rng = np.random.default_rng(stage)
+    B = 300
+    lens = rng.integers(0, 60, size=B)
+    off = np.zeros(B + 1, np.int64)
+    np.cumsum(lens, out=off[1:])
+    tab = (0.01 * rng.standard_normal((509, 64))).astype(np.float32)
+    mt = _Mat([tab], [gi.BF16], seeds=[77])
+    try:
+        mt.m.mfet_set_option(mt.h, mt.m.OPT_STAGE_IDS, stage)
+        ids = rng.integers(0, 2**40, size=int(off[-1]), dtype=np.uint64)
+        w = rng.random(ids.size).astype(np.float32)
+        for pool in (0, 2):
+            got = forward(mt, B, 1, [0], [0], [pool], ids, off, w)
+            ref = orc.embedding_bag(mt.oracle_tables, B, 1, [0], [0], [pool], ids, off, w)
+            assert_close(got, ref, "stage %d pool %d" % (stage, pool))
+    finally:
+        mt.close()
+
+
+@pytest.mark.parametrize("tile", [8, 16, 0])
+def test_many_tiles_per_slot_at_full_batch(tile):
+    """Workload 3 at its full batch over small tables, cut into many more tiles than the GPU
+    keeps resident: whole output against the oracle for two batches in a row, and the bits of
+    the first batch repeat."""
+    w = gi.make_workload(3, rows_scale=2e-4, batch_scale=1.0)
+    b0, b1 = gi.make_batch(w, 0), gi.make_batch(w, 1)
+    with DeviceTables(w.tables) as dt:
+        if tile:
+            dt.m.mfet_set_option(dt.h, dt.m.OPT_TILE, tile)
+        first = workload_forward(dt, w, b0)
+        assert_close(first, workload_oracle(dt, w, b0), "first call")
+        second = workload_forward(dt, w, b1)
+        assert_close(second, workload_oracle(dt, w, b1), "second call")
+        again = workload_forward(dt, w, b0)
+        assert np.array_equal(first.view(np.uint32), again.view(np.uint32))
+
+
 def test_overlapping_launches_give_the_same_bits():
     """MFET_OPT_OVERLAP_LAUNCHES: back-to-back forward calls on one stream, into the same output buffer
     and into different ones, with a consumer kernel between them; every result has the bits of the
