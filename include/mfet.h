@@ -64,7 +64,9 @@ enum {
 
 /* Bits of the device error word (mfet_query_status). */
 enum {
-  MFET_DEV_ROW_RANGE = 1u,      /* a pre-hashed row index was >= rows; skipped */
+  MFET_DEV_ROW_RANGE = 1u,      /* a pre-hashed row index was >= rows: the lookup is skipped for a
+                                   table in device memory, and counts as the table's last row for a
+                                   table in host memory and in mfet_embedding_bag_backward        */
   MFET_DEV_OFFSETS = 2u,        /* offsets decreased inside a bag; bag skipped */
   MFET_DEV_CAPACITY = 4u        /* a host-path batch exceeded the workspace    */
 };
@@ -337,6 +339,25 @@ MFET_API int mfet_profile_read(mfet_tables_t* t, float* stage_ms /*host float[3]
  * stream and copies two counters out of the workspace. Errors: INVALID_ARG, WORKSPACE
  * (no workspace attached), CUDA. */
 MFET_API int mfet_host_path_counts(mfet_tables_t* t, int64_t* n_unique /*host*/, int64_t* n_miss /*host*/);
+
+/* The intermediate results of the most recent host-table slot that ran (paper, Section 3.3
+ * motivates them: only distinct rows that the GPU does not already hold should leave host
+ * memory): its distinct rows in ascending order, for each of them where the row is found
+ * (src[j] >= 0: that slot of the HBM cache; src[j] < 0: entry -1 - src[j] of the list of rows
+ * fetched from host memory), and that list, `miss_rows`, ascending. Counts as returned by
+ * mfet_host_path_counts. uniq dev i64[capacity], src dev i32[capacity], miss_rows dev
+ * i64[capacity]; any of them may be NULL. Waits for the internal streams and for the copies.
+ * Errors: INVALID_ARG (capacity smaller than a count), WORKSPACE (none attached), CUDA. */
+MFET_API int mfet_host_path_result(mfet_tables_t* t, int64_t* uniq, int32_t* src, int64_t* miss_rows,
+                          int64_t capacity);
+
+/* dst[m, :] = row rows[m] of host table `table_id`, m < n: the zero-copy read of listed rows
+ * from the registered host memory (paper, Section 3.3: the largest tables stay in host
+ * memory), as the lookup path issues it for the rows that miss the cache. rows dev i64[n],
+ * each in [0, table rows); dst dev [n, row bytes], 16-byte aligned. Asynchronous on `stream`.
+ * Errors: INVALID_ARG (not a host table, ...), NOT_REGISTERED, ALIGNMENT, CUDA. */
+MFET_API int mfet_host_fetch_rows(mfet_tables_t* t, int32_t table_id, const int64_t* rows, int64_t n, void* dst,
+                         mfet_stream_t stream);
 
 /* Version tag of a table set (paper, Section 3.3 and Algorithm 2: embeddings travel with the
  * version id of the tables that produced them, so that they are scored by the matching

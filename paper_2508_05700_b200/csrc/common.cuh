@@ -50,6 +50,7 @@ struct mfet_tables {
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   cudaEvent_t ev_dedup[2] = {nullptr, nullptr}, ev_fetch[2] = {nullptr, nullptr};  // per result set
   int last_set = 0;              // result set of the most recent host-table batch
+  uint64_t last_row_bytes = 16;  // row bytes that laid out the workspace for it
   void* ws = nullptr;
   uint64_t ws_bytes = 0;
   int64_t ws_max_ids = 0;

@@ -128,6 +128,7 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
     if (prof) cudaEventRecord(t->prof_ev[2], t->fetch);
     if (cudaEventRecord(t->ev_fetch[set], t->fetch) != cudaSuccess) return MFET_ERR_CUDA;
     t->last_set = set;
+    t->last_row_bytes = tb.row_bytes;
   }
   if (!(stage & 2)) return MFET_OK;
 
@@ -226,6 +227,54 @@ int mfet_host_path_counts(mfet_tables_t* t, int64_t* n_unique, int64_t* n_miss) 
   *n_unique = c[0];
   *n_miss = c[1 + (t->last_set & 1)];
   return MFET_OK;
+}
+
+int mfet_host_path_result(mfet_tables_t* t, int64_t* uniq, int32_t* src, int64_t* miss_rows, int64_t capacity) {
+  if (!t || capacity < 0) return MFET_ERR_INVALID_ARG;
+  if (!t->ws) return MFET_ERR_WORKSPACE;
+  WsLayout L;
+  workspace_layout(t->ws_max_ids, t->last_row_bytes, &L);
+  int prev = 0;
+  if (cudaGetDevice(&prev) != cudaSuccess) return MFET_ERR_CUDA;
+  if (prev != t->device && cudaSetDevice(t->device) != cudaSuccess) return MFET_ERR_CUDA;
+  const uint8_t* ws = static_cast<const uint8_t*>(t->ws);
+  const int set = t->last_set & 1;
+  int64_t c[3] = {0, 0, 0};  // n_unique, n_miss of result set 0, of result set 1
+  bool ok = cudaStreamSynchronize(t->side) == cudaSuccess && cudaStreamSynchronize(t->fetch) == cudaSuccess &&
+            cudaMemcpy(c, ws + L.counters, sizeof(c), cudaMemcpyDeviceToHost) == cudaSuccess;
+  int rc = MFET_OK;
+  if (ok && (c[0] > capacity || c[1 + set] > capacity)) rc = MFET_ERR_INVALID_ARG;
+  if (ok && rc == MFET_OK) {
+    if (uniq && c[0] > 0) ok = ok && cudaMemcpy(uniq, ws + L.uniq, (size_t)c[0] * 8, cudaMemcpyDeviceToDevice) == cudaSuccess;
+    if (src && c[0] > 0)
+      ok = ok && cudaMemcpy(src, ws + (set ? L.src2 : L.src), (size_t)c[0] * 4, cudaMemcpyDeviceToDevice) == cudaSuccess;
+    if (miss_rows && c[1 + set] > 0)
+      ok = ok && cudaMemcpy(miss_rows, ws + (set ? L.miss_rows2 : L.miss_rows), (size_t)c[1 + set] * 8,
+                            cudaMemcpyDeviceToDevice) == cudaSuccess;
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+  }
+  if (prev != t->device) cudaSetDevice(prev);
+  if (!ok) return MFET_ERR_CUDA;
+  return rc;
+}
+
+int mfet_host_fetch_rows(mfet_tables_t* t, int32_t table_id, const int64_t* rows, int64_t n, void* dst,
+                         mfet_stream_t stream_) {
+  if (!t || n < 0 || table_id < 0 || table_id >= (int32_t)t->tables.size()) return MFET_ERR_INVALID_ARG;
+  const TableHost& tb = t->tables[(size_t)table_id];
+  if (tb.desc.location != MFET_LOC_HOST) return MFET_ERR_INVALID_ARG;
+  if (!tb.registered) return MFET_ERR_NOT_REGISTERED;
+  if (n == 0) return MFET_OK;
+  if (!rows || !dst) return MFET_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(dst) & 15u) return MFET_ERR_ALIGNMENT;
+  int prev = 0;
+  if (cudaGetDevice(&prev) != cudaSuccess) return MFET_ERR_CUDA;
+  if (prev != t->device && cudaSetDevice(t->device) != cudaSuccess) return MFET_ERR_CUDA;
+  const bool ok = launch_fetch(tb.dev_ptr, tb.stride, (uint32_t)(tb.row_bytes / 16), rows, nullptr, n,
+                               static_cast<uint8_t*>(dst), (cudaStream_t)stream_) == cudaSuccess;
+  if (ok) t->launches += 1;
+  if (prev != t->device) cudaSetDevice(prev);
+  return ok ? MFET_OK : MFET_ERR_CUDA;
 }
 
 int mfet_cache_bytes(const mfet_tables_t* t, int32_t table_id, int64_t n, uint64_t* bytes) {

@@ -38,6 +38,7 @@ EXPORTS = [
     "mfet_embedding_bag_forward_host", "mfet_table_fill", "mfet_query_status", "mfet_set_option",
     "mfet_launch_count", "mfet_status_string", "mfet_dedup_rows_static", "mfet_profile_read", "mfet_host_path_counts", "mfet_tables_set_version", "mfet_tables_version",
     "mfet_host_prefetch", "mfet_embedding_bag_backward", "mfet_embedding_bag_forward_host_async",
+    "mfet_host_path_result", "mfet_host_fetch_rows",
 ]
 BATCH_IDS_ARE_ROWS, BATCH_PREFETCHED = 1, 2
 STATIC_DEDUP_MAX_IDS = 262144
@@ -85,6 +86,8 @@ _lib.mfet_query_status.argtypes = [_P, C.POINTER(C.c_uint32), C.c_int32]
 _lib.mfet_set_option.argtypes = [_P, C.c_int32, C.c_int64]
 _lib.mfet_profile_read.argtypes = [_P, C.POINTER(C.c_float)]
 _lib.mfet_host_path_counts.argtypes = [_P, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+_lib.mfet_host_path_result.argtypes = [_P, _P, _P, _P, C.c_int64]
+_lib.mfet_host_fetch_rows.argtypes = [_P, C.c_int32, _P, C.c_int64, _P, _P]
 _lib.mfet_tables_set_version.argtypes = [_P, C.c_uint64]
 _lib.mfet_tables_version.argtypes = [_P, C.POINTER(C.c_uint64)]
 _lib.mfet_host_prefetch.argtypes = [_P, C.POINTER(BatchShape), _P, _P, _P, _P]
@@ -253,6 +256,14 @@ def mfet_host_path_counts(h):
     a, b = C.c_int64(), C.c_int64()
     _check(_lib.mfet_host_path_counts(h, C.byref(a), C.byref(b)), "mfet_host_path_counts")
     return int(a.value), int(b.value)
+
+
+def mfet_host_path_result(h, uniq, src, miss_rows, capacity: int) -> None:
+    _check(_lib.mfet_host_path_result(h, _ptr(uniq), _ptr(src), _ptr(miss_rows), capacity), "mfet_host_path_result")
+
+
+def mfet_host_fetch_rows(h, table_id: int, rows, n: int, dst, stream=None) -> None:
+    _check(_lib.mfet_host_fetch_rows(h, table_id, _ptr(rows), n, _ptr(dst), _ptr(stream)), "mfet_host_fetch_rows")
 
 
 def mfet_tables_set_version(h, version: int) -> None:

@@ -483,11 +483,19 @@ def test_forward_host_equals_forward():
 
 @pytest.mark.parametrize("n,hi", [(0, 10), (1, 10), (2, 2), (255, 10**9), (256, 10**9), (257, 50), (2047, 10**9),
                                   (2048, 3), (2049, 10**6), (4096, 1), (65537, 10**9), (300_000, 10**9),
-                                  (300_000, 2**62), (100_000, 70_000)])
+                                  (300_000, 2**62), (100_000, 70_000), (8191, 2**33), (8192, 2**22), (8193, 2**11),
+                                  (16 * 512 * 3 + 5, 2047), (1_040_384, 10**9), (1_040_385, 10**9), (1_300_000, 2**40),
+                                  (524_289, 2**34 + 3)])
 def test_dedup_bit_exact(n, hi):
+    """Sizes around the sort's tile boundaries and up to 1.3 million IDs, keys of 1 to 62 bits; a
+    third of the values repeat a few hot rows the way Zipf-distributed IDs do."""
     m = mfet()
     rng = np.random.default_rng(n + hi % 97)
     rows = rng.integers(0, hi, size=n, dtype=np.int64)
+    if n > 16:
+        hot = rng.integers(0, hi, size=5, dtype=np.int64)
+        pick = rng.random(n) < 0.33
+        rows[pick] = hot[rng.integers(0, 5, size=int(pick.sum()))]
     dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
     h = m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), 8, 4, m.F32, m.LOC_DEVICE, 0, 0, 0)])
     try:
@@ -558,6 +566,126 @@ def test_host_table_path_matches_oracle_and_hbm_placement(pinned_by_caller):
     assert_close(hbm, ref)
     assert np.array_equal(hbm[:, 64:], cold[:, 64:])
     assert_close(hbm[:, :64], cold[:, :64])
+
+
+@pytest.mark.parametrize("cache_share", [0.0, 0.02, 1.0])
+def test_cache_probe_and_miss_list_against_a_host_computation(cache_share):
+    """The host-table slot's intermediate results, read back: distinct rows = numpy's sorted unique
+    of the hashed rows; a distinct row has a cache slot exactly when it is in the cache list, and
+    that slot holds it; the miss list is the ascending complement; the fetched rows and the cached
+    rows are the table's rows, bit for bit."""
+    w = gi.make_workload(5, rows_scale=0.001, batch_scale=0.25)
+    b = gi.make_batch(w, 3)
+    n_host = int(b.offsets[w.batch] - b.offsets[0])
+    with DeviceTables(w.tables) as dt:
+        m = dt.m
+        cap = n_host + 64
+        dt.set_workspace(cap)
+        rows_total = w.tables[0].rows
+        cached = np.zeros(0, np.int64)
+        if cache_share >= 1.0:
+            cached = np.arange(rows_total, dtype=np.int64)
+        elif cache_share > 0:
+            cached = _hot_rows(dt, w, 0, 0, int(rows_total * cache_share), rows_total)
+        if cached.size:
+            dt.build_cache(0, cached)
+        got = workload_forward(dt, w, b)
+        assert_close(got, workload_oracle(dt, w, b))
+        n_unique, n_miss = m.mfet_host_path_counts(dt.h)
+        uniq = torch.full((cap,), -1, dtype=torch.int64, device="cuda")
+        src = torch.full((cap,), 0x7FFFFFFF, dtype=torch.int32, device="cuda")
+        miss = torch.full((cap,), -1, dtype=torch.int64, device="cuda")
+        m.mfet_host_path_result(dt.h, uniq, src, miss, cap)
+        want_rows = orc.hash_ids(b.ids[:n_host], w.tables[0].hash_seed, rows_total)
+        want_uniq = np.unique(want_rows)
+        assert n_unique == want_uniq.size
+        uniq, src, miss = uniq.cpu().numpy(), src.cpu().numpy(), miss.cpu().numpy()
+        assert np.array_equal(uniq[:n_unique], want_uniq)
+        assert (uniq[n_unique:] == -1).all() and (src[n_unique:] == 0x7FFFFFFF).all()
+        in_cache = np.isin(want_uniq, cached)
+        assert np.array_equal(src[:n_unique] >= 0, in_cache)
+        assert np.array_equal(cached[src[:n_unique][in_cache]], want_uniq[in_cache])
+        want_miss = want_uniq[~in_cache]
+        assert n_miss == want_miss.size
+        assert np.array_equal(miss[:n_miss], want_miss) and (miss[n_miss:] == -1).all()
+        assert np.array_equal(-1 - src[:n_unique][~in_cache], np.arange(n_miss))
+        # the fetch of listed rows, by itself: the rows of the host table, bit for bit
+        if n_miss:
+            rb = m.row_bytes(w.tables[0].dim, w.tables[0].dtype)
+            dst = torch.zeros(n_miss * rb + 16, dtype=torch.uint8, device="cuda")
+            m.mfet_host_fetch_rows(dt.h, 0, torch.from_numpy(want_miss).cuda(), n_miss, dst, _stream())
+            torch.cuda.synchronize()
+            host = dt.mem[0].numpy().reshape(rows_total, rb)
+            assert np.array_equal(dst.cpu().numpy()[:n_miss * rb].reshape(n_miss, rb), host[want_miss])
+            assert not dst.cpu().numpy()[n_miss * rb:].any()
+        with pytest.raises(m.MfetError):
+            m.mfet_host_path_result(dt.h, None, None, None, max(0, n_unique - 1))
+        with pytest.raises(m.MfetError):
+            m.mfet_host_fetch_rows(dt.h, 1, miss, 1, miss)  # table 1 is not a host table
+
+
+def test_bad_prehashed_row_on_the_host_table_path_counts_as_the_last_row():
+    """A caller-given row index beyond the table, on a slot whose table is in host memory: the error
+    bit is set and the lookup reads the table's last row (documented; a device-memory table skips it)."""
+    rows, dim = 64, 8
+    spec = gi.TableSpec(rows, dim, gi.F16, 0, 0x77, gi.LOC_HOST)
+    with DeviceTables([spec]) as dt:
+        m = dt.m
+        dt.set_workspace(64)
+        ids = np.array([3, 999, 5, 63], np.uint64)
+        off = np.array([0, 3, 4], np.int64)
+        shape, keep = m.make_shape(2, 1, [0], ids_are_rows=True)
+        out = torch.full((2, dim), float("nan"), dtype=torch.float32, device="cuda")
+        m.mfet_embedding_bag_forward(dt.h, shape, torch.from_numpy(ids.view(np.int64)).cuda(),
+                                     torch.from_numpy(off).cuda(), None, [0], [0], out, _stream())
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(dt.h, clear=True) == m.DEV_ROW_RANGE
+        ok_ids = np.array([3, 63, 5, 63], np.uint64)
+        ref = orc.embedding_bag(dt.oracle_tables, 2, 1, [0], [0], [0], ok_ids, off, None, ids_are_rows=True)
+        assert_close(out.cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("dtype,dim", [(gi.BF16, 64), (gi.F32, 8)])
+def test_tables_of_more_than_2_to_32_rows(dtype, dim):
+    """Row indices that need more than 32 bits: a table declared with 2^32 + 1000 rows whose data
+    pointer is placed so that rows 2^32 - 500 ... 2^32 + 999 fall into a small buffer; the batch
+    gives row indices directly. SUM and WSUM (the staging then also holds weights and the upper
+    index halves) against the oracle."""
+    m = mfet()
+    rows = 2**32 + 1000
+    r0, n_real = 2**32 - 500, 1500
+    key = 0xC0FFEE
+    rb = m.row_bytes(dim, dtype)
+    buf = torch.zeros(n_real * rb, dtype=torch.uint8, device="cuda")
+    base = buf.data_ptr() - r0 * rb
+    m.mfet_table_fill(base, r0, n_real, dim, dtype, 0, key, m.VAL_NORMAL, _stream())
+    h = m.mfet_tables_create([m.TableDesc(base, rows, dim, dtype, m.LOC_DEVICE, 0, 0, 0)])
+    try:
+        rng = np.random.default_rng(dim)
+        B = 200
+        lens = rng.integers(0, 30, size=B)
+        lens[7] = 150  # a whole-warp bag
+        off = np.zeros(B + 1, np.int64)
+        np.cumsum(lens, out=off[1:])
+        ids = (r0 + rng.integers(0, n_real, size=int(off[-1]))).astype(np.uint64)
+        wts = rng.random(ids.size).astype(np.float32)
+        otab = [orc.Table(rows=rows, dim=dim, dtype=dtype, hash_seed=0, value_key=key)]
+        shape, keep = m.make_shape(B, 1, [0], ids_are_rows=True)
+        d_ids, d_off, d_w = torch.from_numpy(ids.view(np.int64)).cuda(), torch.from_numpy(off).cuda(), torch.from_numpy(wts).cuda()
+        for pool in (0, 2):
+            out = torch.full((B, dim), float("nan"), dtype=torch.float32, device="cuda")
+            m.mfet_embedding_bag_forward(h, shape, d_ids, d_off, d_w, [0], [pool], out, _stream())
+            torch.cuda.synchronize()
+            assert m.mfet_query_status(h) == 0
+            ref = orc.embedding_bag(otab, B, 1, [0], [0], [pool], ids, off, wts, ids_are_rows=True)
+            assert_close(out.cpu().numpy(), ref, "pool %d" % pool)
+        bad = ids.copy()
+        bad[5] = rows + 3  # beyond the table: skipped, error bit
+        m.mfet_embedding_bag_forward(h, shape, torch.from_numpy(bad.view(np.int64)).cuda(), d_off, d_w, [0], [0], out, _stream())
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(h, clear=True) == m.DEV_ROW_RANGE
+    finally:
+        m.mfet_tables_destroy(h)
 
 
 def test_host_slot_over_workspace_capacity_sets_error_bit():

@@ -6,13 +6,15 @@ request thread that must never trigger the device-wide synchronisation that
 cudaMalloc/cudaFree imply. For them the library carries a small fixed scratch array
 of its own. This test calls that entry point through the C-ABI twice in a row (the
 second call reuses the array with the first call's leftovers in it) and requires the
-very same bits as mfet_dedup_rows, which sorts in a caller-provided workspace.
-The file name makes pytest collect it after every other test.
+very same bits as mfet_dedup_rows, which sorts in a caller-provided workspace, and as
+the CPU checker's sorted-unique definition (so the two GPU entry points cannot drift
+together unnoticed). The file name makes pytest collect it after every other test.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle as orc
 from tests.helpers import mfet
 
 pytestmark = pytest.mark.gpu
@@ -58,6 +60,10 @@ def test_static_dedup_matches_workspace_dedup_on_two_calls_in_a_row():
         assert k == k_ref
         assert np.array_equal(uniq[:k].cpu().numpy(), uniq_ref)  # integer work: bit-exact
         assert np.array_equal(inv[:n].cpu().numpy(), inv_ref)
+        want_uniq, want_inv = orc.dedup(rows[:n].cpu().numpy())
+        assert k == want_uniq.size
+        assert np.array_equal(uniq_ref, want_uniq)
+        assert np.array_equal(inv_ref, want_inv)
 
 
 def test_static_dedup_rejects_sizes_beyond_its_array():
