@@ -1,33 +1,134 @@
 // K-backward: gradient of the pooled output with respect to the rows of one slot's
 // table, as a sparse list (ascending distinct rows + one fp32 gradient vector each).
 // The lookups of the slot are hashed and sorted by row with the dedup machinery; every
-// distinct row then sums coef * grad_out[bag] over its run of lookups in input order
-// (the sort is stable), so the result does not depend on timing.
+// distinct row then sums coef * grad_out[bag] over its run of lookups (the sort is stable:
+// a run is in input order), long runs in pieces that are combined in a fixed order, so the
+// result does not depend on timing.
 #include <cstring>
 
 #include "common.cuh"
 
 using namespace mfet;
 
+static constexpr int32_t kBwdChunkDefault = 256;  // most sorted lookups per warp of the gradient pass
+
 namespace mfet {
 
 namespace {
 
-constexpr int kBwdRegs = 4;  // gradient columns per lane per pass (32 lanes x 4 = 128 columns)
+constexpr int kBwdRegs = 4;      // gradient columns per lane per pass (32 lanes x 4 = 128 columns)
+constexpr int kBwdBatch = 8;     // gradient rows that a warp requests together
 
-// One warp per distinct row u: its run is sorted positions [seg_start[u], seg_start[u+1])
-// (or n for the last row). For every lookup of the run: find its bag by bisection in the
-// feature's offsets, take coef = 1 (SUM), 1/len (MEAN) or weights[i] (WSUM), and add
-// coef * grad_out[bag, col + d]. Lanes own columns d = lane, lane + 32, ...
-__global__ void __launch_bounds__(256) backward_rows_kernel(const uint32_t* __restrict__ sorted_pos,
-                                                            const int32_t* __restrict__ seg_start,
-                                                            const int64_t* __restrict__ n_unique, NSrc ns,
-                                                            const int64_t* __restrict__ offsets_f, int32_t batch,
-                                                            const float* __restrict__ weights, int32_t pooling,
-                                                            const float* __restrict__ grad_out, int64_t out_ld,
-                                                            uint32_t col, uint32_t dim, float* __restrict__ grad_vals) {
+// The lookups of the slot, sorted by table row (stably, so a row's run is in input order), are
+// cut into CHUNKS of `chunk` consecutive sorted positions, one warp per chunk; a hot row's run of
+// thousands of lookups is thereby spread over many warps instead of being one warp's serial loop.
+// Inside a chunk the warp works on 32 lookups at a time: every lane finds the bag of one lookup
+// (bisection in the feature's offsets) and its coefficient - 1 (SUM), 1/len (MEAN) or weights[i]
+// (WSUM) -, then the 32 lookups are added one after the other, lanes owning the columns
+// d = lane, lane + 32, ... of grad_out[bag, col + d]. A row whose run lies inside the chunk is
+// stored directly. A run that crosses a chunk boundary leaves a partial sum in the chunk's HEAD
+// slot (the run began before the chunk) or TAIL slot (it goes on after it);
+// backward_combine_kernel adds the partial sums of such a row in chunk order. The order of the
+// additions depends only on the inputs and the chunk length.
+__global__ void __launch_bounds__(256) backward_chunks_kernel(const uint32_t* __restrict__ sorted_pos,
+                                                              const int32_t* __restrict__ inverse,
+                                                              const int32_t* __restrict__ seg_start,
+                                                              const int64_t* __restrict__ n_unique, NSrc ns,
+                                                              const int64_t* __restrict__ offsets_f, int32_t batch,
+                                                              const float* __restrict__ weights, int32_t pooling,
+                                                              const float* __restrict__ grad_out, int64_t out_ld,
+                                                              uint32_t col, uint32_t dim, int32_t chunk,
+                                                              float* __restrict__ partial, float* __restrict__ grad_vals) {
   const int64_t feat_lo = offsets_f[0];
   int64_t n = offsets_f[batch] - feat_lo;
+  if (n < 0 || n > ns.cap) n = 0;
+  const int64_t nu = *n_unique;
+  const int lane = threadIdx.x & 31;
+  const int64_t k = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;  // this warp's chunk
+  const int64_t c0 = k * chunk;
+  if (c0 >= n) return;
+  const int64_t c1 = c0 + chunk < n ? c0 + chunk : n;
+  float* head = partial + (size_t)(2 * k) * dim;
+  float* tail = head + dim;
+  for (uint32_t d0 = 0; d0 < dim; d0 += 32 * kBwdRegs) {
+    float acc[kBwdRegs];
+#pragma unroll
+    for (int r = 0; r < kBwdRegs; ++r) acc[r] = 0.f;
+    int32_t cur = -1;  // distinct-row index of the run that acc belongs to
+    auto flush = [&](int32_t u) {
+      // run of row u: sorted positions [j0, j1)
+      const int64_t j0 = seg_start[u];
+      const int64_t j1 = ((int64_t)u + 1 < nu) ? (int64_t)seg_start[u + 1] : n;
+      float* dst = (j0 >= c0 && j1 <= c1) ? grad_vals + (size_t)u * dim : (j0 < c0 ? head : tail);
+#pragma unroll
+      for (int r = 0; r < kBwdRegs; ++r) {
+        const uint32_t d = d0 + lane + 32 * r;
+        if (d < dim) dst[d] = acc[r];
+        acc[r] = 0.f;
+      }
+    };
+    for (int64_t j32 = c0; j32 < c1; j32 += 32) {
+      // every lane: one lookup's row, bag and coefficient
+      const int64_t j = j32 + lane;
+      int32_t u = -1, bag = 0;
+      float coef = 0.f;
+      if (j < c1) {
+        const uint32_t pos = sorted_pos[j];
+        const int64_t i = feat_lo + pos;  // position of the lookup in ids / weights
+        u = inverse[pos];
+        int lo = 0, hi = batch;  // the last b with offsets_f[b] <= i
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (offsets_f[mid] <= i) lo = mid;
+          else hi = mid;
+        }
+        bag = lo;
+        coef = 1.f;
+        if (pooling == MFET_POOL_MEAN) coef = __fdiv_rn(1.f, (float)(offsets_f[lo + 1] - offsets_f[lo]));
+        else if (pooling == MFET_POOL_WSUM) coef = weights[i];
+      }
+      const int cnt = (int)(c1 - j32 < 32 ? c1 - j32 : 32);
+      for (int t0 = 0; t0 < cnt; t0 += kBwdBatch) {
+        float g[kBwdBatch][kBwdRegs];
+#pragma unroll
+        for (int t = 0; t < kBwdBatch; ++t) {  // the loads of a batch do not depend on one another
+          const int32_t bt = __shfl_sync(0xFFFFFFFFu, bag, (t0 + t) & 31);
+          const float* row = grad_out + (int64_t)bt * out_ld + col + d0;
+#pragma unroll
+          for (int r = 0; r < kBwdRegs; ++r) {
+            const uint32_t d = d0 + lane + 32 * r;
+            g[t][r] = (t0 + t < cnt && d < dim) ? __ldg(row + lane + 32 * r) : 0.f;
+          }
+        }
+#pragma unroll
+        for (int t = 0; t < kBwdBatch; ++t) {
+          const int32_t ut = __shfl_sync(0xFFFFFFFFu, u, (t0 + t) & 31);
+          const float ct = __shfl_sync(0xFFFFFFFFu, coef, (t0 + t) & 31);
+          if (t0 + t < cnt) {
+            if (ut != cur) {
+              if (cur >= 0) flush(cur);
+              cur = ut;
+            }
+#pragma unroll
+            for (int r = 0; r < kBwdRegs; ++r) acc[r] = fmaf(ct, g[t][r], acc[r]);
+          }
+        }
+      }
+    }
+    if (cur >= 0) flush(cur);
+  }
+}
+
+// One warp per distinct row whose run crosses a chunk boundary: its gradient is the TAIL slot of
+// the chunk where the run begins, the HEAD slots of the chunks it covers entirely, and the HEAD
+// slot of the chunk where it ends, added in that order.
+__global__ void __launch_bounds__(256) backward_combine_kernel(const int32_t* __restrict__ seg_start,
+                                                               const int64_t* __restrict__ n_unique, NSrc ns,
+                                                               const int64_t* __restrict__ offsets_f, int32_t batch,
+                                                               uint32_t dim, int32_t chunk,
+                                                               const float* __restrict__ partial,
+                                                               float* __restrict__ grad_vals) {
+  int64_t n = offsets_f[batch] - offsets_f[0];
   if (n < 0 || n > ns.cap) n = 0;
   const int64_t nu = *n_unique;
   const int lane = threadIdx.x & 31;
@@ -35,46 +136,33 @@ __global__ void __launch_bounds__(256) backward_rows_kernel(const uint32_t* __re
   for (int64_t u = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < nu; u += warps) {
     const int64_t j0 = seg_start[u];
     const int64_t j1 = (u + 1 < nu) ? (int64_t)seg_start[u + 1] : n;
-    for (uint32_t d0 = 0; d0 < dim; d0 += 32 * kBwdRegs) {
-      float acc[kBwdRegs];
-#pragma unroll
-      for (int k = 0; k < kBwdRegs; ++k) acc[k] = 0.f;
-      for (int64_t j = j0; j < j1; ++j) {
-        const int64_t i = feat_lo + sorted_pos[j];  // position of the lookup in ids / weights
-        // bag of i: the last b with offsets_f[b] <= i
-        int lo = 0, hi = batch;
-        while (hi - lo > 1) {
-          const int mid = (lo + hi) >> 1;
-          if (offsets_f[mid] <= i) lo = mid;
-          else hi = mid;
-        }
-        float coef = 1.f;
-        if (pooling == MFET_POOL_MEAN) coef = __fdiv_rn(1.f, (float)(offsets_f[lo + 1] - offsets_f[lo]));
-        else if (pooling == MFET_POOL_WSUM) coef = weights[i];
-        const float* g = grad_out + (int64_t)lo * out_ld + col + d0;
-#pragma unroll
-        for (int k = 0; k < kBwdRegs; ++k) {
-          const uint32_t d = d0 + lane + 32 * k;
-          if (d < dim) acc[k] = fmaf(coef, g[lane + 32 * k], acc[k]);
-        }
-      }
-#pragma unroll
-      for (int k = 0; k < kBwdRegs; ++k) {
-        const uint32_t d = d0 + lane + 32 * k;
-        if (d < dim) grad_vals[u * dim + d] = acc[k];
-      }
+    const int64_t k0 = j0 / chunk, k1 = (j1 - 1) / chunk;
+    if (k0 == k1) continue;  // stored directly by the chunk's warp
+    for (uint32_t d = lane; d < dim; d += 32) {
+      float s = partial[(size_t)(2 * k0 + 1) * dim + d];
+      for (int64_t k = k0 + 1; k <= k1; ++k) s += partial[(size_t)(2 * k) * dim + d];
+      grad_vals[(size_t)u * dim + d] = s;
     }
   }
 }
 
 }  // namespace
 
-cudaError_t launch_backward(const uint32_t* sorted_pos, const int32_t* seg_start, const int64_t* n_unique, NSrc ns,
-                            const int64_t* offsets_f, int32_t batch, const float* weights, int32_t pooling,
-                            const float* grad_out, int64_t out_ld, uint32_t col, uint32_t dim, float* grad_vals,
-                            cudaStream_t s) {
-  backward_rows_kernel<<<sm_count() * 8, 256, 0, s>>>(sorted_pos, seg_start, n_unique, ns, offsets_f, batch, weights, pooling,
-                                               grad_out, out_ld, col, dim, grad_vals);
+// partial: room for 2 * dim floats per chunk of `chunk` sorted lookups, capacity ns.cap lookups.
+cudaError_t launch_backward(const uint32_t* sorted_pos, const int32_t* inverse, const int32_t* seg_start,
+                            const int64_t* n_unique, NSrc ns, const int64_t* offsets_f, int32_t batch,
+                            const float* weights, int32_t pooling, const float* grad_out, int64_t out_ld, uint32_t col,
+                            uint32_t dim, int32_t chunk, float* partial, float* grad_vals, cudaStream_t s) {
+  const int64_t chunks = (ns.cap + chunk - 1) / chunk;
+  const int64_t blocks = (chunks + 7) / 8;  // 8 warps per block, one chunk per warp
+  if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
+  backward_chunks_kernel<<<(unsigned)(blocks > 0 ? blocks : 1), 256, 0, s>>>(
+      sorted_pos, inverse, seg_start, n_unique, ns, offsets_f, batch, weights, pooling, grad_out, out_ld, col, dim, chunk,
+      partial, grad_vals);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  backward_combine_kernel<<<sm_count() * 8, 256, 0, s>>>(seg_start, n_unique, ns, offsets_f, batch, dim, chunk, partial,
+                                                         grad_vals);
   return cudaGetLastError();
 }
 
@@ -128,11 +216,26 @@ extern "C" int mfet_embedding_bag_backward(mfet_tables_t* t, const mfet_batch_sh
   a.sorted_pos_out = &sorted_pos;
   int rc = MFET_OK;
   if (launch_dedup(a, &t->launches, stream) != cudaSuccess) rc = MFET_ERR_CUDA;
+  // partial sums of runs that cross a chunk boundary go to the part of the workspace that the
+  // sort does not use (from the miss list to the end): two vectors per chunk; a workspace too
+  // small for that (tiny capacities) gets one chunk = one warp for everything
+  float* partial = reinterpret_cast<float*>(ws + Lw.miss_rows);
+  const uint64_t room = Lw.total - Lw.miss_rows;
+  // short chunks spread the work over more warps; the shortest whose partial sums fit is taken
+  int32_t chunk = 64;
+  auto fits = [&](int32_t c) {
+    return ((uint64_t)(t->ws_max_ids + c - 1) / c) * 2ull * tb.desc.dim * sizeof(float) <= room;
+  };
+  while (chunk < kBwdChunkDefault && !fits(chunk)) chunk *= 2;
+  if (!fits(chunk)) {
+    if (t->ws_max_ids > 0x7FFFFFE0LL) rc = MFET_ERR_WORKSPACE;
+    else chunk = (int32_t)((t->ws_max_ids + 31) / 32 * 32);  // every run lies inside the one chunk: no partial sums
+  }
   if (rc == MFET_OK &&
-      launch_backward(sorted_pos, a.src, n_rows, a.ns, offsets + (int64_t)f * B, B, weights, pooling[slot], grad_out,
-                      out_ld, (uint32_t)col, tb.desc.dim, grad_vals, stream) != cudaSuccess)
+      launch_backward(sorted_pos, a.inverse, a.src, n_rows, a.ns, offsets + (int64_t)f * B, B, weights, pooling[slot],
+                      grad_out, out_ld, (uint32_t)col, tb.desc.dim, chunk, partial, grad_vals, stream) != cudaSuccess)
     rc = MFET_ERR_CUDA;
-  if (rc == MFET_OK) t->launches += 1;
+  if (rc == MFET_OK) t->launches += 2;
   if (prev != t->device) cudaSetDevice(prev);
   return rc;
 }

@@ -240,10 +240,10 @@ cudaError_t launch_bag_indirect(const BagParams& p, const IndirectParams& ip, cu
 int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, int32_t feature, int32_t pooling,
                   uint32_t col, cudaStream_t side, int stage, int set);
 
-cudaError_t launch_backward(const uint32_t* sorted_pos, const int32_t* seg_start, const int64_t* n_unique, NSrc ns,
-                            const int64_t* offsets_f, int32_t batch, const float* weights, int32_t pooling,
-                            const float* grad_out, int64_t out_ld, uint32_t col, uint32_t dim, float* grad_vals,
-                            cudaStream_t s);
+cudaError_t launch_backward(const uint32_t* sorted_pos, const int32_t* inverse, const int32_t* seg_start,
+                            const int64_t* n_unique, NSrc ns, const int64_t* offsets_f, int32_t batch,
+                            const float* weights, int32_t pooling, const float* grad_out, int64_t out_ld, uint32_t col,
+                            uint32_t dim, int32_t chunk, float* partial, float* grad_vals, cudaStream_t s);
 
 // launch helpers implemented in the kernel files
 cudaError_t launch_hash(const uint64_t* ids, int64_t n, uint64_t seed, uint64_t rows, uint64_t magic,

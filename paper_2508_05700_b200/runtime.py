@@ -76,14 +76,14 @@ class LookupEngine:
         ids = gi.hot_ids(self.w, feature, count)
         d = torch.from_numpy(ids.view(np.int64)).cuda(self.device)
         m.mfet_hash_ids(self.h, table_id, d, d.numel(), d, self.stream)
-        # first occurrence of every row in popularity order (plain tensor plumbing, not the lookup path)
-        uniq, inv = torch.unique(d, return_inverse=True)
-        first = torch.full((uniq.numel(),), d.numel(), dtype=torch.int64, device=d.device)
-        first.scatter_reduce_(0, inv, torch.arange(d.numel(), device=d.device), reduce="amin")
-        if uniq.numel() > want:
-            keep = torch.topk(first, want, largest=False).indices
-            uniq = uniq[keep]
-        rows_sorted = torch.sort(uniq).values.cpu().numpy()
+        rows = d.cpu().numpy()
+        del d
+        # the first `want` distinct rows in popularity order, ascending (host-side set-up, numpy)
+        uniq, first = np.unique(rows, return_index=True)
+        if uniq.size > want:
+            bound = np.partition(first, want - 1)[want - 1]
+            uniq = uniq[first <= bound]
+        rows_sorted = np.ascontiguousarray(uniq, dtype=np.int64)
         nbytes = m.mfet_cache_bytes(self.h, table_id, rows_sorted.size)
         mem = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda:%d" % self.device)
         m.mfet_cache_build(self.h, table_id, rows_sorted, mem, mem.numel(), self.stream)

@@ -58,3 +58,48 @@ def test_backward_matches_oracle(config, rows_scale, batch_scale):
                 assert np.isfinite(got).all()
                 assert (err <= 1e-6 + 1e-5 * mass[got_rows]).all(), float((err / (1e-6 + 1e-5 * mass[got_rows])).max())
             col += t.dim
+
+
+@pytest.mark.parametrize("B,max_len,rows,dim,pool", [(300, 40, 7, 136, 2), (300, 40, 1, 8, 1), (3, 4, 5, 264, 0),
+                                                    (64, 300, 3, 32, 0)])
+def test_backward_hot_rows_and_tiny_workspaces(B, max_len, rows, dim, pool):
+    """A few rows that receive hundreds or thousands of lookups each (their runs are summed in pieces
+    by many warps and combined), more than 128 columns, and a workspace too small to hold partial
+    sums (then one warp sums everything): the sparse gradient against the oracle's dense scatter-add."""
+    m = mfet()
+    rng = np.random.default_rng(B * 1000 + dim)
+    spec = gi.TableSpec(rows, dim, gi.F32, 0x5EED, 0x1234)
+    lens = rng.integers(0, max_len + 1, size=B)
+    off = np.zeros(B + 1, np.int64)
+    np.cumsum(lens, out=off[1:])
+    n = int(off[-1])
+    ids = rng.integers(0, 2**40, size=n, dtype=np.uint64)
+    wts = rng.random(n).astype(np.float32)
+    gout = (0.01 * rng.standard_normal((B, dim))).astype(np.float32)
+    with DeviceTables([spec]) as dt:
+        dt.set_workspace(max(n, 1))
+        shape, keep = m.make_shape(B, 1, [0])
+        g_rows = torch.full((max(n, 1),), -1, dtype=torch.int64, device="cuda")
+        g_vals = torch.full((max(n, 1), dim), float("nan"), dtype=torch.float32, device="cuda")
+        nr = torch.zeros(1, dtype=torch.int64, device="cuda")
+        d_ids = torch.from_numpy(ids.view(np.int64)).cuda() if n else torch.zeros(1, dtype=torch.int64, device="cuda")
+        m.mfet_embedding_bag_backward(dt.h, shape, d_ids, torch.from_numpy(off).cuda(), torch.from_numpy(wts).cuda()
+                                      if n else torch.zeros(1, device="cuda"), [0], [pool], torch.from_numpy(gout).cuda(),
+                                      0, g_rows, g_vals, nr, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(dt.h) == 0
+        k = int(nr.item())
+        got_rows, got = g_rows[:k].cpu().numpy(), g_vals[:k].cpu().numpy().astype(np.float64)
+        ref = orc.embedding_bag_backward_slot(dt.oracle_tables, B, [0], [0], [pool], 0, dim, 0, ids, off, wts, gout)
+        mass = orc.embedding_bag_backward_slot(dt.oracle_tables, B, [0], [0], [pool], 0, dim, 0, ids, off, wts,
+                                               np.abs(gout))
+        assert np.array_equal(got_rows, np.unique(orc.hash_ids(ids, spec.hash_seed, rows)))
+        err = np.abs(got - ref[got_rows])
+        assert np.isfinite(got).all()
+        assert (err <= 1e-6 + 1e-5 * mass[got_rows]).all(), float((err / (1e-6 + 1e-5 * mass[got_rows])).max())
+        again = torch.full_like(g_vals, float("nan"))
+        m.mfet_embedding_bag_backward(dt.h, shape, d_ids, torch.from_numpy(off).cuda(), torch.from_numpy(wts).cuda()
+                                      if n else torch.zeros(1, device="cuda"), [0], [pool], torch.from_numpy(gout).cuda(),
+                                      0, g_rows, again, nr, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert torch.equal(again[:k], g_vals[:k])  # the order of the additions is fixed
