@@ -68,7 +68,9 @@ enum {
                                    table in device memory, and counts as the table's last row for a
                                    table in host memory and in mfet_embedding_bag_backward        */
   MFET_DEV_OFFSETS = 2u,        /* offsets decreased inside a bag; bag skipped */
-  MFET_DEV_CAPACITY = 4u        /* a host-path batch exceeded the workspace    */
+  MFET_DEV_CAPACITY = 4u,       /* a host-path batch exceeded the workspace    */
+  MFET_DEV_BOUNDS = 8u          /* only in the bounds-checked build of the library: a kernel formed an
+                                   index outside its array; the access was skipped               */
 };
 
 /* One embedding table. Rows are `dim` elements of `dtype`, row-major.

@@ -354,6 +354,7 @@ int mfet_host_prefetch(mfet_tables_t* t, const mfet_batch_shape_t* shape, const 
   p.offsets = offsets;
   p.err = t->err_dev;
   p.batch = B;
+  p.n_features = F;
   p.flags = (uint32_t)(shape->flags & 1);
   // the internal stream starts after what `stream` holds now (the batch's inputs) and is not joined back
   if (cudaEventRecord(t->ev_fork, stream) != cudaSuccess) return MFET_ERR_CUDA;
@@ -416,6 +417,7 @@ int mfet_embedding_bag_forward(mfet_tables_t* t, const mfet_batch_shape_t* shape
   p.err = t->err_dev;
   p.out_ld = out_ld;
   p.batch = B;
+  p.n_features = F;
   p.flags = (uint32_t)(shape->flags & 1);
   if (aligned16(out) && out_ld % 4 == 0) p.flags |= 2u;
   if (t->overlap) p.flags |= 16u;

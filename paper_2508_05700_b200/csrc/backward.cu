@@ -38,7 +38,8 @@ __global__ void __launch_bounds__(256) backward_chunks_kernel(const uint32_t* __
                                                               const float* __restrict__ weights, int32_t pooling,
                                                               const float* __restrict__ grad_out, int64_t out_ld,
                                                               uint32_t col, uint32_t dim, int32_t chunk,
-                                                              float* __restrict__ partial, float* __restrict__ grad_vals) {
+                                                              float* __restrict__ partial, float* __restrict__ grad_vals,
+                                                              uint32_t* err) {
   const int64_t feat_lo = offsets_f[0];
   int64_t n = offsets_f[batch] - feat_lo;
   if (n < 0 || n > ns.cap) n = 0;
@@ -56,6 +57,7 @@ __global__ void __launch_bounds__(256) backward_chunks_kernel(const uint32_t* __
     for (int r = 0; r < kBwdRegs; ++r) acc[r] = 0.f;
     int32_t cur = -1;  // distinct-row index of the run that acc belongs to
     auto flush = [&](int32_t u) {
+      if (!MFET_IN_BOUNDS(err, u >= 0 && (int64_t)u < nu)) return;
       // run of row u: sorted positions [j0, j1)
       const int64_t j0 = seg_start[u];
       const int64_t j1 = ((int64_t)u + 1 < nu) ? (int64_t)seg_start[u + 1] : n;
@@ -73,7 +75,8 @@ __global__ void __launch_bounds__(256) backward_chunks_kernel(const uint32_t* __
       int32_t u = -1, bag = 0;
       float coef = 0.f;
       if (j < c1) {
-        const uint32_t pos = sorted_pos[j];
+        uint32_t pos = sorted_pos[j];
+        if (!MFET_IN_BOUNDS(err, (int64_t)pos < n)) pos = 0;
         const int64_t i = feat_lo + pos;  // position of the lookup in ids / weights
         u = inverse[pos];
         int lo = 0, hi = batch;  // the last b with offsets_f[b] <= i
@@ -152,13 +155,14 @@ __global__ void __launch_bounds__(256) backward_combine_kernel(const int32_t* __
 cudaError_t launch_backward(const uint32_t* sorted_pos, const int32_t* inverse, const int32_t* seg_start,
                             const int64_t* n_unique, NSrc ns, const int64_t* offsets_f, int32_t batch,
                             const float* weights, int32_t pooling, const float* grad_out, int64_t out_ld, uint32_t col,
-                            uint32_t dim, int32_t chunk, float* partial, float* grad_vals, cudaStream_t s) {
+                            uint32_t dim, int32_t chunk, float* partial, float* grad_vals, uint32_t* err,
+                            cudaStream_t s) {
   const int64_t chunks = (ns.cap + chunk - 1) / chunk;
   const int64_t blocks = (chunks + 7) / 8;  // 8 warps per block, one chunk per warp
   if (blocks > 0x7FFFFFFF) return cudaErrorInvalidValue;
   backward_chunks_kernel<<<(unsigned)(blocks > 0 ? blocks : 1), 256, 0, s>>>(
       sorted_pos, inverse, seg_start, n_unique, ns, offsets_f, batch, weights, pooling, grad_out, out_ld, col, dim, chunk,
-      partial, grad_vals);
+      partial, grad_vals, err);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   backward_combine_kernel<<<sm_count() * 8, 256, 0, s>>>(seg_start, n_unique, ns, offsets_f, batch, dim, chunk, partial,
@@ -233,7 +237,8 @@ extern "C" int mfet_embedding_bag_backward(mfet_tables_t* t, const mfet_batch_sh
   }
   if (rc == MFET_OK &&
       launch_backward(sorted_pos, a.inverse, a.src, n_rows, a.ns, offsets + (int64_t)f * B, B, weights, pooling[slot],
-                      grad_out, out_ld, (uint32_t)col, tb.desc.dim, chunk, partial, grad_vals, stream) != cudaSuccess)
+                      grad_out, out_ld, (uint32_t)col, tb.desc.dim, chunk, partial, grad_vals, t->err_dev,
+                      stream) != cudaSuccess)
     rc = MFET_ERR_CUDA;
   if (rc == MFET_OK) t->launches += 2;
   if (prev != t->device) cudaSetDevice(prev);

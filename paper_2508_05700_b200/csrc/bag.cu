@@ -172,6 +172,20 @@ struct RowAddr {
   uint64_t stride;
   uint32_t stride32;
   bool wide;              // row index or stride beyond 32 bits
+#ifdef MFET_CHECKED
+  uint64_t rows, rows2;   // rows of the table (IND: of the cache), IND: of the fetched-rows buffer
+  uint32_t* err;
+  __device__ __forceinline__ bool row_ok(uint32_t lo, uint32_t hi) const {
+    if constexpr (IND) {
+      const bool cached = (int32_t)lo >= 0;
+      return MFET_IN_BOUNDS(err, (uint64_t)(cached ? lo : ~lo) < (cached ? rows : rows2));
+    } else {
+      return MFET_IN_BOUNDS(err, (wide ? (((uint64_t)hi << 32) | lo) : (uint64_t)lo) < rows);
+    }
+  }
+#else
+  __device__ __forceinline__ bool row_ok(uint32_t, uint32_t) const { return true; }
+#endif
   // the common case: row index and stride fit 32 bits
   __device__ __forceinline__ void get_narrow(uint32_t lo, const uint8_t*& chunk, const uint8_t*& meta) const {
     if constexpr (IND) {
@@ -217,14 +231,18 @@ __device__ __forceinline__ void run_steps(const uint32_t* srow, const uint32_t* 
       if (j < left && chunk_ok) {
         const uint32_t lo = srow[j * GG];
         const uint32_t hi = (!IND && ra.wide) ? shi[j * GG] : 0u;
-        if (IND || (ra.wide ? (lo & hi) != 0xFFFFFFFFu : lo != 0xFFFFFFFFu)) {
+        if ((IND || (ra.wide ? (lo & hi) != 0xFFFFFFFFu : lo != 0xFFFFFFFFu)) && ra.row_ok(lo, hi)) {
           ra.get(lo, hi, a, m);
           v[j] = load_chunk<DT>(a, m);
         }
       }
     } else {
-      ra.get_narrow(srow[j * GG], a, m);
-      v[j] = load_chunk<DT>(a, m);
+      const uint32_t lo = srow[j * GG];
+      v[j] = make_uint4(0u, 0u, 0u, 0u);
+      if (ra.row_ok(lo, 0u)) {
+        ra.get_narrow(lo, a, m);
+        v[j] = load_chunk<DT>(a, m);
+      }
     }
   }
 #pragma unroll
@@ -321,6 +339,7 @@ __device__ __forceinline__ void pool_bag(const BagParams& p, const SlotDev& s, c
   ReduceScatter<E, 0, GG, LPR>::run(a, sub, off, writer);
   if (!writer) return;
   const int bi = bag & 0xFF;
+  if (!MFET_IN_BOUNDS(p.err, w.b0 + bi < p.batch && (int64_t)s.col_off + c * E + off + NF <= p.out_ld)) return;
   float* o = p.out + (int64_t)(w.b0 + bi) * p.out_ld + s.col_off + c * E + off;
   if (bag & kNotFirst) {
 #pragma unroll
@@ -373,6 +392,11 @@ __device__ __forceinline__ void pool_window(const BagParams& p, const SlotDev& s
     ra.stride = ip.row_bytes;
     ra.stride32 = (uint32_t)ip.row_bytes;
     ra.wide = false;
+#ifdef MFET_CHECKED
+    ra.rows = (uint64_t)ip.cache_n;
+    ra.rows2 = (uint64_t)ip.cap;
+    ra.err = p.err;
+#endif
   } else {
     ra.tbase = s.table + coff;
     ra.mbase = s.table + s.meta_off;
@@ -380,6 +404,11 @@ __device__ __forceinline__ void pool_window(const BagParams& p, const SlotDev& s
     ra.stride = s.stride;
     ra.stride32 = (uint32_t)s.stride;
     ra.wide = s.narrow == 0;
+#ifdef MFET_CHECKED
+    ra.rows = s.rows;
+    ra.rows2 = 0;
+    ra.err = p.err;
+#endif
   }
   const int n_long = BPW > 1 ? w.n_long : 0;
   while (true) {
@@ -444,7 +473,14 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
   float* sw = reinterpret_cast<float*>(dyn + ((p.flags & 4u) ? C : 0));
   uint32_t* shi = dyn + ((p.flags & 8u) ? ((p.flags & 4u) ? 2 * C : C) : 0);
   const long long* offs = reinterpret_cast<const long long*>(p.offsets) + (int64_t)s.feature * p.batch;
-  if (tid <= nb) soff[tid] = __ldcs(offs + b0 + tid);
+  if (tid <= nb) {
+    soff[tid] = MFET_IN_BOUNDS(p.err, (int64_t)s.feature * p.batch + b0 + tid <= (int64_t)p.n_features * p.batch)
+                    ? __ldcs(offs + b0 + tid) : 0;
+  }
+#ifdef MFET_CHECKED
+  __shared__ int64_t snnz;  // number of IDs in the batch: the extent of ids and weights
+  if (tid == 0) snnz = p.offsets[(int64_t)p.n_features * p.batch];
+#endif
   if (IND && tid < 2) sfeat[tid] = offs[tid ? p.batch : 0];
   if (tid < kCnt) (&scnt[0][0])[tid] = 0;
   if (tid == 255) snext = 0;
@@ -474,8 +510,9 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
 
   // the ID (IND: the position in the dedup list) of a lookup -> staged value of window position pos
   auto stage = [&](int pos, uint64_t id) {
+    if (!MFET_IN_BOUNDS(p.err, pos >= 0 && pos < C)) return;
     if constexpr (IND) {
-      srow[pos] = (uint32_t)__ldg(ip.src + (uint32_t)id);
+      srow[pos] = MFET_IN_BOUNDS(p.err, (int64_t)(uint32_t)id < ip.cap) ? (uint32_t)__ldg(ip.src + (uint32_t)id) : 0u;
     } else {
       uint64_t row = mod_rows(splitmix64(id ^ s.seed), s.rows, s.magic);
       if (pre) {  // the caller's row indices are used as they are, and checked
@@ -489,9 +526,25 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
       if (wide) shi[pos] = (uint32_t)(row >> 32);
     }
   };
+#ifdef MFET_CHECKED
+  const int64_t nnz = snnz;
+#endif
   auto fetch_id = [&](int64_t i) -> uint64_t {
-    if constexpr (IND) return (uint32_t)__ldg(ip.inverse + (i - feat_lo));
-    else return __ldcs(ids + i);
+    if constexpr (IND) {
+      if (!MFET_IN_BOUNDS(p.err, i - feat_lo >= 0 && i - feat_lo < ip.cap)) return 0;
+      return (uint32_t)__ldg(ip.inverse + (i - feat_lo));
+    } else {
+#ifdef MFET_CHECKED
+      if (!MFET_IN_BOUNDS(p.err, i >= 0 && i < nnz)) return 0;
+#endif
+      return __ldcs(ids + i);
+    }
+  };
+  auto fetch_w = [&](int64_t i) -> float {
+#ifdef MFET_CHECKED
+    if (!MFET_IN_BOUNDS(p.err, i >= 0 && i < nnz)) return 0.f;
+#endif
+    return __ldcs(p.weights + i);
   };
 
   for (int64_t w0 = 0;; w0 += C) {
@@ -507,7 +560,7 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
       ew[k] = 1.f;
       if (pos < wn) {
         eid[k] = fetch_id(g0 + pos);
-        if (wsum) ew[k] = __ldcs(p.weights + g0 + pos);
+        if (wsum) ew[k] = fetch_w(g0 + pos);
       }
     }
     // ---- order the bags that have a piece in this window: the long pieces first (a whole
@@ -580,7 +633,7 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
       const int pos = tid + k * 256;
       if (pos < wn) {
         stage(pos, eid[k]);
-        if (wsum) sw[pos] = ew[k];
+        if (wsum && MFET_IN_BOUNDS(p.err, pos < C)) sw[pos] = ew[k];
       }
     }
     // the rest of a large window, again with the loads of a batch requested before any of them is used
@@ -590,7 +643,7 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
         const int pos = base + k * 256;
         if (pos < wn) {
           eid[k] = fetch_id(g0 + pos);
-          if (wsum) ew[k] = __ldcs(p.weights + g0 + pos);
+          if (wsum) ew[k] = fetch_w(g0 + pos);
         }
       }
 #pragma unroll
@@ -598,7 +651,7 @@ __device__ __forceinline__ void bag_body(const BagParams& p, const IndirectParam
         const int pos = base + k * 256;
         if (pos < wn) {
           stage(pos, eid[k]);
-          if (wsum) sw[pos] = ew[k];
+          if (wsum && MFET_IN_BOUNDS(p.err, pos < C)) sw[pos] = ew[k];
         }
       }
     }

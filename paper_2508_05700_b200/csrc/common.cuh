@@ -113,11 +113,23 @@ struct BagParams {
                          // bit4: the launch may begin before the stream's previous kernel has finished
   int32_t group_policy;  // 0 auto, 1 one row-group per bag, 2 one warp per bag
   int32_t stage_cap;     // IDs staged per window, 32 .. kStageMax (0: default)
+  int32_t n_features;    // offsets has n_features * batch + 1 entries (used by the bounds-checked build)
   SlotDev slot[kMaxSlotsPerLaunch];
 };
 static_assert(sizeof(BagParams) <= 4000, "BagParams must fit the kernel parameter space");
 
 // ---------------------------------------------------------- device helpers --
+
+// Bounds-checked build (-DMFET_CHECKED, `python -m paper_2508_05700_b200.build --checked`): every
+// index that a kernel forms from the caller's data or from its own arithmetic is tested against
+// the extent of the array right before the access; a violation sets MFET_DEV_BOUNDS in the device
+// error word and the access is skipped (no trap, no assert: the context stays usable). The normal
+// build compiles the tests away.
+#ifdef MFET_CHECKED
+#define MFET_IN_BOUNDS(err, cond) ((cond) ? true : (atomicOr((err), (uint32_t)MFET_DEV_BOUNDS), false))
+#else
+#define MFET_IN_BOUNDS(err, cond) true
+#endif
 
 // splitmix64 output function (public domain; Steele, Lea, Flood).
 __host__ __device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
@@ -223,6 +235,7 @@ struct IndirectParams {
   const uint8_t* staging;
   uint64_t row_bytes;
   int64_t cap;
+  int64_t cache_n;            // rows in the cache (used by the bounds-checked build)
 };
 
 struct CacheLayout {
@@ -233,8 +246,10 @@ struct CacheLayout {
 uint64_t workspace_layout(int64_t max_ids, uint64_t max_row_bytes, WsLayout* L);
 void cache_layout(uint64_t rows, int64_t n, uint64_t row_bytes, CacheLayout* L);
 cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s);
+// table_rows, cap: the table's rows and the capacity (in rows) of rows_list / dst, for the bounds-checked build
 cudaError_t launch_fetch(const uint8_t* table, uint64_t stride, uint32_t chunks, const int64_t* rows_list,
-                         const int64_t* n_ptr, int64_t n_imm, uint8_t* dst, cudaStream_t s);
+                         const int64_t* n_ptr, int64_t n_imm, uint8_t* dst, uint64_t table_rows, int64_t cap,
+                         uint32_t* err, cudaStream_t s);
 cudaError_t launch_bag_indirect(const BagParams& p, const IndirectParams& ip, cudaStream_t s);
 // stage bit0: hash + dedup + probe + fetch into result set `set`; bit1: pool from it
 int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, int32_t feature, int32_t pooling,
@@ -243,7 +258,8 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
 cudaError_t launch_backward(const uint32_t* sorted_pos, const int32_t* inverse, const int32_t* seg_start,
                             const int64_t* n_unique, NSrc ns, const int64_t* offsets_f, int32_t batch,
                             const float* weights, int32_t pooling, const float* grad_out, int64_t out_ld, uint32_t col,
-                            uint32_t dim, int32_t chunk, float* partial, float* grad_vals, cudaStream_t s);
+                            uint32_t dim, int32_t chunk, float* partial, float* grad_vals, uint32_t* err,
+                            cudaStream_t s);
 
 // launch helpers implemented in the kernel files
 cudaError_t launch_hash(const uint64_t* ids, int64_t n, uint64_t seed, uint64_t rows, uint64_t magic,

@@ -162,7 +162,8 @@ __global__ void __launch_bounds__(kSortThreads) scatter_kernel(NSrc ns, const ui
                                                                const uint32_t* __restrict__ idx_in,
                                                                uint64_t* __restrict__ keys_out,
                                                                uint32_t* __restrict__ idx_out, int shift,
-                                                               const uint32_t* __restrict__ hist, int nblk) {
+                                                               const uint32_t* __restrict__ hist, int nblk,
+                                                               uint32_t* err) {
   constexpr int kWarps = kSortThreads / 32;
   __shared__ uint16_t wcnt[kSortRounds][kWarps][256];  // counts, then offsets inside the tile (< 2048)
   int64_t lo;
@@ -220,8 +221,10 @@ __global__ void __launch_bounds__(kSortThreads) scatter_kernel(NSrc ns, const ui
     if (dr[r] >> 16) {
       const uint32_t d = dr[r] & 255u;
       const uint32_t pos = sbase[d] + wcnt[r][warp][d] + ((dr[r] >> 8) & 255u);
-      keys_out[pos] = k[r];
-      idx_out[pos] = src[r];
+      if (MFET_IN_BOUNDS(err, (int64_t)pos < n)) {
+        keys_out[pos] = k[r];
+        idx_out[pos] = src[r];
+      }
     }
   }
 }
@@ -333,7 +336,8 @@ __global__ void __launch_bounds__(kScanThreads) unique_write_kernel(NSrc ns, con
                                                                     const int32_t* __restrict__ probe_tmp,
                                                                     const uint32_t* __restrict__ tile_counts, int nblk,
                                                                     int64_t* __restrict__ uniq, int32_t* __restrict__ inverse,
-                                                                    int32_t* __restrict__ src, int64_t* __restrict__ miss_rows) {
+                                                                    int32_t* __restrict__ src, int64_t* __restrict__ miss_rows,
+                                                                    uint32_t* err) {
   __shared__ uint32_t sh[8];
   int64_t lo;
   const int64_t n = resolve_n(ns, &lo);
@@ -368,7 +372,7 @@ __global__ void __launch_bounds__(kScanThreads) unique_write_kernel(NSrc ns, con
 #pragma unroll
   for (int j = 0; j < kScanItems; ++j) {
     const int64_t i = i0 + j;
-    if (i < n) {
+    if (i < n && MFET_IN_BOUNDS(err, (int64_t)u - (head[j] ? 0 : 1) < n && (int64_t)m <= n && (int64_t)idx[i] < n)) {
       if (head[j]) {
         uniq[u] = (int64_t)k[j];
         if (!PROBE && src) src[u] = (int32_t)i;  // where this row's run starts in the sorted order
@@ -460,7 +464,7 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
                                                       a.hash->magic, a.hash->pre_hashed, shift, hist, nblk, a.err, tickets);
     else
       hist_kernel<false><<<nblk, kSortThreads, 0, s>>>(a.ns, kin, nullptr, nullptr, 0, 0, 0, 0, shift, hist, nblk, a.err, tickets);
-    scatter_kernel<<<nblk, kSortThreads, 0, s>>>(a.ns, kin, iin, kout, iout, shift, hist, nblk);
+    scatter_kernel<<<nblk, kSortThreads, 0, s>>>(a.ns, kin, iin, kout, iout, shift, hist, nblk, a.err);
     *launches += 2;
     // next pass reads what this one wrote
     kin = kout;
@@ -474,13 +478,13 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
     unique_count_kernel<true><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, *a.cache, probe_tmp, tile_counts, nblk2,
                                                              tickets + 1, a.n_unique, a.n_miss);
     unique_write_kernel<true><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, iin, probe_tmp, tile_counts, nblk2, a.uniq,
-                                                            a.inverse, a.src, a.miss_rows);
+                                                            a.inverse, a.src, a.miss_rows, a.err);
   } else {
     CacheDev none{};
     unique_count_kernel<false><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, none, nullptr, tile_counts, nblk2, tickets + 1,
                                                               a.n_unique, nullptr);
     unique_write_kernel<false><<<nblk2, kScanThreads, 0, s>>>(a.ns, kin, iin, nullptr, tile_counts, nblk2, a.uniq,
-                                                             a.inverse, a.src, nullptr);
+                                                             a.inverse, a.src, nullptr, a.err);
   }
   if (a.sorted_pos_out) *a.sorted_pos_out = iin;
   *launches += 2;

@@ -22,8 +22,10 @@ constexpr int kFetchUnroll = 4;
 __global__ void __launch_bounds__(256) fetch_rows_kernel(const uint8_t* __restrict__ table, uint64_t stride,
                                                          uint32_t chunks, const int64_t* __restrict__ rows_list,
                                                          const int64_t* __restrict__ n_ptr, int64_t n_imm,
-                                                         uint8_t* __restrict__ dst) {
-  const int64_t n = n_ptr ? *n_ptr : n_imm;
+                                                         uint8_t* __restrict__ dst, uint64_t table_rows, int64_t cap,
+                                                         uint32_t* err) {
+  int64_t n = n_ptr ? *n_ptr : n_imm;
+  if (!MFET_IN_BOUNDS(err, n >= 0 && n <= cap)) n = 0;
   const int64_t total = n * chunks;
   const int64_t step = (int64_t)gridDim.x * blockDim.x;
   for (int64_t q0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; q0 < total; q0 += step * kFetchUnroll) {
@@ -34,7 +36,9 @@ __global__ void __launch_bounds__(256) fetch_rows_kernel(const uint8_t* __restri
       if (q < total) {
         const int64_t m = q / chunks;
         const uint32_t c = (uint32_t)(q - m * chunks);
-        v[k] = ld_row16(table + (uint64_t)rows_list[m] * stride + (uint64_t)c * 16);
+        const uint64_t row = (uint64_t)rows_list[m];
+        v[k] = MFET_IN_BOUNDS(err, row < table_rows) ? ld_row16(table + row * stride + (uint64_t)c * 16)
+                                                     : make_uint4(0u, 0u, 0u, 0u);
       }
     }
 #pragma unroll
@@ -64,8 +68,10 @@ __global__ void __launch_bounds__(256) cache_index_kernel(const int64_t* __restr
 }  // namespace
 
 cudaError_t launch_fetch(const uint8_t* table, uint64_t stride, uint32_t chunks, const int64_t* rows_list,
-                         const int64_t* n_ptr, int64_t n_imm, uint8_t* dst, cudaStream_t s) {
-  fetch_rows_kernel<<<sm_count() * 4, 256, 0, s>>>(table, stride, chunks, rows_list, n_ptr, n_imm, dst);
+                         const int64_t* n_ptr, int64_t n_imm, uint8_t* dst, uint64_t table_rows, int64_t cap,
+                         uint32_t* err, cudaStream_t s) {
+  fetch_rows_kernel<<<sm_count() * 4, 256, 0, s>>>(table, stride, chunks, rows_list, n_ptr, n_imm, dst, table_rows, cap,
+                                                   err);
   return cudaGetLastError();
 }
 
@@ -122,7 +128,8 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
     if (prof) cudaEventRecord(t->prof_ev[1], side);
     if (cudaEventRecord(t->ev_dedup[set], side) != cudaSuccess) return MFET_ERR_CUDA;
     if (cudaStreamWaitEvent(t->fetch, t->ev_dedup[set], 0) != cudaSuccess) return MFET_ERR_CUDA;
-    if (launch_fetch(tb.dev_ptr, tb.stride, chunks, a.miss_rows, a.n_miss, 0, staging, t->fetch) != cudaSuccess)
+    if (launch_fetch(tb.dev_ptr, tb.stride, chunks, a.miss_rows, a.n_miss, 0, staging, tb.desc.rows, t->ws_max_ids,
+                     t->err_dev, t->fetch) != cudaSuccess)
       return MFET_ERR_CUDA;
     t->launches += 1;
     if (prof) cudaEventRecord(t->prof_ev[2], t->fetch);
@@ -135,7 +142,7 @@ int run_host_slot(mfet_tables* t, const TableHost& tb, const BagParams& base, in
   // the pooling follows on the side stream once the set's rows have arrived; a later dedup into the
   // same set is behind it in that stream
   if (cudaStreamWaitEvent(side, t->ev_fetch[set], 0) != cudaSuccess) return MFET_ERR_CUDA;
-  IndirectParams ip{a.inverse, a.src, tb.cache.data, staging, tb.row_bytes, t->ws_max_ids};
+  IndirectParams ip{a.inverse, a.src, tb.cache.data, staging, tb.row_bytes, t->ws_max_ids, tb.cache.n};
   BagParams p = base;
   p.flags &= ~1u;  // the indirect path never hashes
   p.flags |= base.flags & 2u;
@@ -271,7 +278,8 @@ int mfet_host_fetch_rows(mfet_tables_t* t, int32_t table_id, const int64_t* rows
   if (cudaGetDevice(&prev) != cudaSuccess) return MFET_ERR_CUDA;
   if (prev != t->device && cudaSetDevice(t->device) != cudaSuccess) return MFET_ERR_CUDA;
   const bool ok = launch_fetch(tb.dev_ptr, tb.stride, (uint32_t)(tb.row_bytes / 16), rows, nullptr, n,
-                               static_cast<uint8_t*>(dst), (cudaStream_t)stream_) == cudaSuccess;
+                               static_cast<uint8_t*>(dst), tb.desc.rows, n, t->err_dev,
+                               (cudaStream_t)stream_) == cudaSuccess;
   if (ok) t->launches += 1;
   if (prev != t->device) cudaSetDevice(prev);
   return ok ? MFET_OK : MFET_ERR_CUDA;
@@ -320,7 +328,7 @@ int mfet_cache_build(mfet_tables_t* t, int32_t table_id, const int64_t* rows_sor
     ok = cudaGetLastError() == cudaSuccess;
   }
   ok = ok && launch_fetch(tb.dev_ptr, tb.stride, (uint32_t)(tb.row_bytes / 16), keys, nullptr, n, mem + L.data,
-                          stream) == cudaSuccess;
+                          tb.desc.rows, n, t->err_dev, stream) == cudaSuccess;
   ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
   if (ok) {
     t->launches += 2;

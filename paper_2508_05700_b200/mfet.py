@@ -15,7 +15,8 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmfet.so")
+# MFET_LIBRARY selects another build of the same library (the bounds-checked one, libmfet_checked.so)
+LIB_PATH = os.environ.get("MFET_LIBRARY") or os.path.join(_HERE, "libmfet.so")
 
 F32, F16, BF16, INT4 = 0, 1, 2, 3
 POOL_SUM, POOL_MEAN, POOL_WSUM = 0, 1, 2
@@ -29,7 +30,7 @@ OPT_OVERLAP_LAUNCHES = 5
 OK = 0
 ERR_INVALID_ARG, ERR_NOT_REGISTERED, ERR_ALIGNMENT, ERR_UNSUPPORTED_DIM = -1, -2, -3, -4
 ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
-DEV_ROW_RANGE, DEV_OFFSETS, DEV_CAPACITY = 1, 2, 4
+DEV_ROW_RANGE, DEV_OFFSETS, DEV_CAPACITY, DEV_BOUNDS = 1, 2, 4, 8
 
 EXPORTS = [
     "mfet_row_bytes", "mfet_tables_create", "mfet_tables_destroy", "mfet_host_tables_register",
