@@ -218,7 +218,7 @@ struct RowAddr {
 // lane has only `left` of the N steps (possibly none or all of them), and a
 // staged row may be the "no row" sentinel or lie outside this lane's chunks;
 // what is not loaded counts as zeros.
-template <int DT, int GG, bool IND, int N, bool PRED, bool WS>
+template <int DT, int GG, bool IND, int N, bool PRED, bool WS, bool PLAIN = false>
 __device__ __forceinline__ void run_steps(const uint32_t* srow, const uint32_t* shi, const float* sw,
                                           const RowAddr<IND>& ra, bool wsum, int left, bool chunk_ok,
                                           unsigned long long* acc) {
@@ -226,7 +226,17 @@ __device__ __forceinline__ void run_steps(const uint32_t* srow, const uint32_t* 
 #pragma unroll
   for (int j = 0; j < N; ++j) {
     const uint8_t *a, *m;
-    if constexpr (PRED) {
+    if constexpr (PRED && PLAIN) {
+      // predicated, but the table is narrow, every staged row is a row and every lane has a chunk
+      v[j] = make_uint4(0u, 0u, 0u, 0u);
+      if (j < left) {
+        const uint32_t lo = srow[j * GG];
+        if (ra.row_ok(lo, 0u)) {
+          ra.get_narrow(lo, a, m);
+          v[j] = load_chunk<DT>(a, m);
+        }
+      }
+    } else if constexpr (PRED) {
       v[j] = make_uint4(0u, 0u, 0u, 0u);
       if (j < left && chunk_ok) {
         const uint32_t lo = srow[j * GG];
@@ -303,9 +313,15 @@ __device__ __forceinline__ void gather_piece(const Win& w, const RowAddr<IND>& r
   if (wsum) t = run_common<DT, GG, IND, true>(srow, sw, ra, min_steps, acc);
   else t = run_common<DT, GG, IND, false>(srow, sw, ra, min_steps, acc);
   // what is left: fewer than 4 common steps and the steps that only some lanes have
-  for (; t < max_steps; t += 4)
-    run_steps<DT, GG, IND, 4, true, false>(srow + t * GG, shi + t * GG, sw + t * GG, ra, wsum, steps - t, chunk_ok,
-                                           acc);
+  if (fast_ok) {
+    for (; t < max_steps; t += 4)
+      run_steps<DT, GG, IND, 4, true, false, true>(srow + t * GG, shi + t * GG, sw + t * GG, ra, wsum, steps - t, true,
+                                                   acc);
+  } else {
+    for (; t < max_steps; t += 4)
+      run_steps<DT, GG, IND, 4, true, false>(srow + t * GG, shi + t * GG, sw + t * GG, ra, wsum, steps - t, chunk_ok,
+                                             acc);
+  }
 }
 
 // Listed bag q of the window (or no bag: q < 0), pooled by a bag group of GG row
