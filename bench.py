@@ -718,12 +718,16 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
                                                 w.pooling, p_out[a], io[a], io_bytes, lanes[a].cuda_stream)
     for j in range(max(4, args.warmup)):
         e2e_step(j)
-    barrier()
-    t_e2e = time.perf_counter()
-    for j in range(args.steps):
-        e2e_step(j)
-    barrier()  # both lanes drained: every result is in host memory
-    e2e_ms = 1e3 * (time.perf_counter() - t_e2e)
+    # the K-step region five times (every region drained: all results in host memory); the median is reported
+    e2e_regions = []
+    for _ in range(5 if world == 1 else 1):
+        barrier()
+        t_e2e = time.perf_counter()
+        for j in range(args.steps):
+            e2e_step(j)
+        barrier()  # both lanes drained: every result is in host memory
+        e2e_regions.append(1e3 * (time.perf_counter() - t_e2e))
+    e2e_ms = float(np.median(e2e_regions))
     t_load1 = time.time()
     clocks = sampler.stop(t_load0, t_load1) if sampler else None
 
@@ -815,7 +819,8 @@ def measure(args, config, rank, world, dist, with_cpu_baseline, sampler_gpu=None
         "e2e": {"value": units / (e2e_ms_all * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 # the two directions of the link run at the same time; the busier one bounds the step
                 "link_gbps": max(h2d, d2h) * args.steps / (e2e_ms_all * 1e-3) / 1e9,  # per GPU
-                "link_direction": "d2h" if d2h >= h2d else "h2d"},
+                "link_direction": "d2h" if d2h >= h2d else "h2d",
+                "regions_ms": [round(x, 3) for x in e2e_regions]},
         "gpu_launches": int(launches),
         "roofline": roofline,
         "pooling_kernel": series,
