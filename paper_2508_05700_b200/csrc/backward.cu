@@ -122,13 +122,15 @@ __global__ void __launch_bounds__(256) backward_chunks_kernel(const uint32_t* __
   }
 }
 
-// One warp per distinct row whose run crosses a chunk boundary: its gradient is the TAIL slot of
-// the chunk where the run begins, the HEAD slots of the chunks it covers entirely, and the HEAD
-// slot of the chunk where it ends, added in that order.
+// Rows whose run crosses a chunk boundary: the gradient is the TAIL slot of the chunk where the run
+// begins, the HEAD slots of the chunks it covers entirely, and the HEAD slot of the chunk where it
+// ends, added in that order. A warp looks at 32 rows at a time (one per lane: most runs lie inside
+// one chunk and need nothing), then works through the ones that do with all its lanes on the
+// columns. chunk = 1 << chunk_shift.
 __global__ void __launch_bounds__(256) backward_combine_kernel(const int32_t* __restrict__ seg_start,
                                                                const int64_t* __restrict__ n_unique, NSrc ns,
                                                                const int64_t* __restrict__ offsets_f, int32_t batch,
-                                                               uint32_t dim, int32_t chunk,
+                                                               uint32_t dim, int32_t chunk_shift,
                                                                const float* __restrict__ partial,
                                                                float* __restrict__ grad_vals) {
   int64_t n = offsets_f[batch] - offsets_f[0];
@@ -136,15 +138,51 @@ __global__ void __launch_bounds__(256) backward_combine_kernel(const int32_t* __
   const int64_t nu = *n_unique;
   const int lane = threadIdx.x & 31;
   const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-  for (int64_t u = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < nu; u += warps) {
-    const int64_t j0 = seg_start[u];
-    const int64_t j1 = (u + 1 < nu) ? (int64_t)seg_start[u + 1] : n;
-    const int64_t k0 = j0 / chunk, k1 = (j1 - 1) / chunk;
-    if (k0 == k1) continue;  // stored directly by the chunk's warp
-    for (uint32_t d = lane; d < dim; d += 32) {
-      float s = partial[(size_t)(2 * k0 + 1) * dim + d];
-      for (int64_t k = k0 + 1; k <= k1; ++k) s += partial[(size_t)(2 * k) * dim + d];
-      grad_vals[(size_t)u * dim + d] = s;
+  for (int64_t u0 = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * 32; u0 < nu; u0 += warps * 32) {
+    const int64_t u = u0 + lane;
+    int64_t k0 = 0, k1 = 0;
+    if (u < nu) {
+      const int64_t j0 = seg_start[u];
+      const int64_t j1 = (u + 1 < nu) ? (int64_t)seg_start[u + 1] : n;
+      k0 = j0 >> chunk_shift;
+      k1 = (j1 - 1) >> chunk_shift;
+    }
+    uint32_t todo = __ballot_sync(0xFFFFFFFFu, k0 != k1);  // runs inside one chunk were stored by the chunk's warp
+    while (todo) {
+      const int t = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const int64_t a0 = __shfl_sync(0xFFFFFFFFu, k0, t), a1 = __shfl_sync(0xFFFFFFFFu, k1, t);
+      // the loads of 8 chunks x 4 column groups are requested together (a hot row spans hundreds of
+      // chunks); the additions of a column stay in chunk order
+      for (uint32_t d0 = 0; d0 < dim; d0 += 32 * kBwdRegs) {
+        float s[kBwdRegs];
+#pragma unroll
+        for (int r = 0; r < kBwdRegs; ++r) {
+          const uint32_t d = d0 + lane + 32 * r;
+          s[r] = d < dim ? partial[(size_t)(2 * a0 + 1) * dim + d] : 0.f;
+        }
+        for (int64_t kb = a0 + 1; kb <= a1; kb += 8) {
+          float v[8][kBwdRegs];
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int r = 0; r < kBwdRegs; ++r) {
+              const uint32_t d = d0 + lane + 32 * r;
+              v[j][r] = (kb + j <= a1 && d < dim) ? __ldcg(partial + (size_t)(2 * (kb + j)) * dim + d) : 0.f;
+            }
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (kb + j <= a1) {
+#pragma unroll
+              for (int r = 0; r < kBwdRegs; ++r) s[r] += v[j][r];
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < kBwdRegs; ++r) {
+          const uint32_t d = d0 + lane + 32 * r;
+          if (d < dim) grad_vals[(size_t)(u0 + t) * dim + d] = s[r];
+        }
+      }
     }
   }
 }
@@ -165,8 +203,13 @@ cudaError_t launch_backward(const uint32_t* sorted_pos, const int32_t* inverse, 
       partial, grad_vals, err);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  backward_combine_kernel<<<sm_count() * 8, 256, 0, s>>>(seg_start, n_unique, ns, offsets_f, batch, dim, chunk, partial,
-                                                         grad_vals);
+  if (chunks <= 1) return cudaSuccess;  // one chunk holds every run: nothing to combine
+  int shift = 0;
+  while ((1 << shift) < chunk) ++shift;  // chunk is a power of two whenever there is more than one
+  int64_t cblocks = (ns.cap + 32 * 8 - 1) / (32 * 8);  // 8 warps per block, 32 rows per warp and round
+  if (cblocks > (int64_t)sm_count() * 8) cblocks = (int64_t)sm_count() * 8;
+  backward_combine_kernel<<<(unsigned)(cblocks > 0 ? cblocks : 1), 256, 0, s>>>(seg_start, n_unique, ns, offsets_f, batch,
+                                                                            dim, shift, partial, grad_vals);
   return cudaGetLastError();
 }
 
@@ -225,8 +268,9 @@ extern "C" int mfet_embedding_bag_backward(mfet_tables_t* t, const mfet_batch_sh
   // small for that (tiny capacities) gets one chunk = one warp for everything
   float* partial = reinterpret_cast<float*>(ws + Lw.miss_rows);
   const uint64_t room = Lw.total - Lw.miss_rows;
-  // short chunks spread the work over more warps; the shortest whose partial sums fit is taken
-  int32_t chunk = 64;
+  // short chunks spread the work over more warps, long ones keep a hot row's list of partial sums short:
+  // 64 lookups per chunk up to 128 k lookups, 256 from 512 k; at least the shortest whose partial sums fit
+  int32_t chunk = t->ws_max_ids > 512 * 1024 ? 256 : (t->ws_max_ids > 128 * 1024 ? 128 : 64);
   auto fits = [&](int32_t c) {
     return ((uint64_t)(t->ws_max_ids + c - 1) / c) * 2ull * tb.desc.dim * sizeof(float) <= room;
   };
