@@ -187,7 +187,9 @@ MFET_API int mfet_host_prefetch(mfet_tables_t* t, const mfet_batch_shape_t* shap
  * as a sparse list: grad_rows = ascending distinct rows that the slot looked up,
  * grad_vals[k, :] = sum over the lookups i of row grad_rows[k] of
  *     c_i * grad_out[b(i), col_slot : col_slot + dim],
- * c_i = 1 (SUM), 1/len(bag) (MEAN) or weights[i] (WSUM), accumulated in fp32 in input order.
+ * c_i = 1 (SUM), 1/len(bag) (MEAN) or weights[i] (WSUM), accumulated in fp32 in an order that depends only
+ * on the inputs and the workspace capacity (a row's lookups in input order, long runs in pieces of 64 to 256
+ * lookups whose partial sums are added in order), so repeated calls give identical bits.
  *   shape, ids, offsets, weights, table_ids, pooling: as in the forward call
  *   grad_out   dev f32[B, out_ld]: gradient of `out`
  *   slot       which slot's table (0 <= slot < L); its table may live in HBM or host memory
