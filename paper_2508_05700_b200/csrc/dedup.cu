@@ -50,51 +50,63 @@ __device__ __forceinline__ bool last_block_arrives(uint32_t* ticket) {
   return last;
 }
 
+// The histogram kernel runs 1024 threads per tile (the scatter kernel 256): the block that arrives
+// last scans tiles x 256 counters, and its critical path is the number of dependent memory round
+// trips of one thread, so four threads share a digit's column.
+constexpr int kHistThreads = 1024;
+constexpr int kHistRounds = kSortTile / kHistThreads;
+constexpr int kHistGroups = kHistThreads / 256;  // threads that share one digit in the scan
+
 // Turns the per-tile digit counts hist[tile][digit] into the global start position of every
 // (digit, tile) pair in digit-major order: start(d, b) = all counts of smaller digits + counts
-// of digit d in tiles before b. Run by the 256 threads of one block; thread d owns digit d, so
-// loads and stores are coalesced across the digits and a thread's loads are independent.
+// of digit d in tiles before b. Run by the 1024 threads of one block: thread (g, d) owns digit d in
+// the g-th quarter of the tiles, so loads and stores are coalesced across the digits, and a
+// thread's loads are independent of one another (batches of 16 are issued together).
 __device__ __forceinline__ void scan_digit_counts(uint32_t* hist, int nblk) {
+  __shared__ uint32_t part[kHistGroups][256];  // keys of digit d in the tiles of group g
+  __shared__ uint32_t dstart[256];             // keys of all smaller digits
   __shared__ uint32_t warp_tot[8];
-  const int d = threadIdx.x;
-  // every load below is independent of the others: batches of 16 are issued together so that
-  // the pass costs nblk/16 memory round trips instead of nblk
+  const int d = threadIdx.x & 255, g = threadIdx.x >> 8;
+  const int per = (nblk + kHistGroups - 1) / kHistGroups;
+  const int b0 = g * per, b1 = min(nblk, b0 + per);
   uint32_t tot = 0;
-  int b = 0;
-  for (; b + 16 <= nblk; b += 16) {
+  for (int b = b0; b < b1; b += 16) {
     uint32_t v[16];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) v[j] = __ldcg(hist + (size_t)(b + j) * 256 + d);
+    for (int j = 0; j < 16; ++j) v[j] = b + j < b1 ? __ldcg(hist + (size_t)(b + j) * 256 + d) : 0u;
 #pragma unroll
     for (int j = 0; j < 16; ++j) tot += v[j];
   }
-  for (; b < nblk; ++b) tot += __ldcg(hist + (size_t)b * 256 + d);
-  const int lane = d & 31;
-  uint32_t inc = tot;
-#pragma unroll
-  for (int k = 1; k < 32; k <<= 1) {
-    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, k);
-    if (lane >= k) inc += t;
-  }
-  if (lane == 31) warp_tot[d >> 5] = inc;
+  part[g][d] = tot;
   __syncthreads();
-  uint32_t run = inc - tot;
+  if (g == 0) {
+    uint32_t all = 0;
+#pragma unroll
+    for (int q = 0; q < kHistGroups; ++q) all += part[q][d];
+    const int lane = d & 31;
+    uint32_t inc = all;
+#pragma unroll
+    for (int k = 1; k < 32; k <<= 1) {
+      const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, inc, k);
+      if (lane >= k) inc += t;
+    }
+    if (lane == 31) warp_tot[d >> 5] = inc;
+    dstart[d] = inc - all;  // exclusive inside the warp; the warps before are added below
+  }
+  __syncthreads();
+  uint32_t run = dstart[d];
   for (int w = 0; w < (d >> 5); ++w) run += warp_tot[w];
-  b = 0;
-  for (; b + 16 <= nblk; b += 16) {
+#pragma unroll
+  for (int q = 0; q < kHistGroups; ++q) run += q < g ? part[q][d] : 0u;
+  for (int b = b0; b < b1; b += 16) {
     uint32_t v[16];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) v[j] = __ldcg(hist + (size_t)(b + j) * 256 + d);
+    for (int j = 0; j < 16; ++j) v[j] = b + j < b1 ? __ldcg(hist + (size_t)(b + j) * 256 + d) : 0u;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      hist[(size_t)(b + j) * 256 + d] = run;
+      if (b + j < b1) hist[(size_t)(b + j) * 256 + d] = run;
       run += v[j];
     }
-  }
-  for (; b < nblk; ++b) {
-    const uint32_t v = __ldcg(hist + (size_t)b * 256 + d);
-    hist[(size_t)b * 256 + d] = run;
-    run += v;
   }
 }
 
@@ -102,7 +114,7 @@ __device__ __forceinline__ void scan_digit_counts(uint32_t* hist, int nblk) {
 // scatter positions. With HASH the keys are produced here from the raw IDs (first pass of
 // a host-table slot) and stored for the later passes.
 template <bool HASH>
-__global__ void __launch_bounds__(kSortThreads) hist_kernel(NSrc ns, const uint64_t* __restrict__ keys_in,
+__global__ void __launch_bounds__(kHistThreads) hist_kernel(NSrc ns, const uint64_t* __restrict__ keys_in,
                                                             uint64_t* __restrict__ keys_store,
                                                             const uint64_t* __restrict__ ids, uint64_t seed,
                                                             uint64_t rows, uint64_t magic, uint32_t pre_hashed,
@@ -116,13 +128,13 @@ __global__ void __launch_bounds__(kSortThreads) hist_kernel(NSrc ns, const uint6
     if (raw < 0) atomicOr(err, (uint32_t)MFET_DEV_OFFSETS);
     if (raw > ns.cap) atomicOr(err, (uint32_t)MFET_DEV_CAPACITY);
   }
-  h[threadIdx.x] = 0;
+  if (threadIdx.x < 256) h[threadIdx.x] = 0;
   __syncthreads();
   const int64_t base = (int64_t)blockIdx.x * kSortTile;
   const int lane = threadIdx.x & 31;
 #pragma unroll
-  for (int r = 0; r < kSortRounds; ++r) {
-    const int64_t i = base + r * kSortThreads + threadIdx.x;
+  for (int r = 0; r < kHistRounds; ++r) {
+    const int64_t i = base + r * kHistThreads + threadIdx.x;
     const bool valid = i < n;
     uint64_t k = 0;
     if (valid) {
@@ -145,7 +157,7 @@ __global__ void __launch_bounds__(kSortThreads) hist_kernel(NSrc ns, const uint6
     if (valid && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&h[d], (uint32_t)__popc(peers));
   }
   __syncthreads();
-  hist[(size_t)blockIdx.x * 256 + threadIdx.x] = h[threadIdx.x];  // block-major: coalesced
+  if (threadIdx.x < 256) hist[(size_t)blockIdx.x * 256 + threadIdx.x] = h[threadIdx.x];  // block-major: coalesced
   if (last_block_arrives(ticket)) {
     scan_digit_counts(hist, nblk);
     if (threadIdx.x == 0) *ticket = 0;  // ready for the next pass
@@ -460,10 +472,10 @@ cudaError_t launch_dedup(const DedupArgs& a, uint64_t* launches, cudaStream_t s)
   for (int p = 0; p < passes; ++p) {
     const int shift = 8 * p;
     if (p == 0 && a.hash)
-      hist_kernel<true><<<nblk, kSortThreads, 0, s>>>(a.ns, nullptr, ka, a.hash->ids, a.hash->seed, a.hash->rows,
+      hist_kernel<true><<<nblk, kHistThreads, 0, s>>>(a.ns, nullptr, ka, a.hash->ids, a.hash->seed, a.hash->rows,
                                                       a.hash->magic, a.hash->pre_hashed, shift, hist, nblk, a.err, tickets);
     else
-      hist_kernel<false><<<nblk, kSortThreads, 0, s>>>(a.ns, kin, nullptr, nullptr, 0, 0, 0, 0, shift, hist, nblk, a.err, tickets);
+      hist_kernel<false><<<nblk, kHistThreads, 0, s>>>(a.ns, kin, nullptr, nullptr, 0, 0, 0, 0, shift, hist, nblk, a.err, tickets);
     scatter_kernel<<<nblk, kSortThreads, 0, s>>>(a.ns, kin, iin, kout, iout, shift, hist, nblk, a.err);
     *launches += 2;
     // next pass reads what this one wrote
