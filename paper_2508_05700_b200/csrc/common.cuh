@@ -139,13 +139,13 @@ __host__ __device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
   return x ^ (x >> 31);
 }
 
-// Exact h mod d for a runtime divisor, with magic = floor((2^64-1)/d).
-// q = floor(h*magic / 2^64) underestimates floor(h/d) by at most 2, so the
-// remainder estimate is below 3d and two conditional subtractions finish it.
+// Exact h mod d for a runtime divisor d >= 1, with magic = floor((2^64-1)/d). Let e = 2^64 - magic*d:
+// 0 < e <= d (e = d exactly when d is a power of two). Then h*magic/2^64 = h/d - h*e/(d*2^64), and the
+// last term lies in [0, 1) because h < 2^64 and e <= d. So q = floor(h*magic / 2^64) is floor(h/d) or
+// one less, the remainder estimate is below 2d, and ONE conditional subtraction finishes it.
 __device__ __forceinline__ uint64_t mod_rows(uint64_t h, uint64_t d, uint64_t magic) {
   uint64_t q = __umul64hi(h, magic);
   uint64_t r = h - q * d;
-  if (r >= d) r -= d;
   if (r >= d) r -= d;
   return r;
 }

@@ -46,6 +46,60 @@ def test_hash_ids_bit_exact(rows):
         m.mfet_tables_destroy(h)
 
 
+def _ids_that_hash_to(values, seed):
+    """Raw IDs whose splitmix64(id ^ seed) is exactly `values`: the generator's output function is a
+    bijection of 64-bit words (xor-shifts and odd multipliers), inverted here step by step in python
+    integers. Test-side only: it lets the test choose the number that goes INTO the modulo."""
+    M = (1 << 64) - 1
+
+    def unshift(y, s):
+        x = y
+        for _ in range(64 // s + 1):
+            x = y ^ (x >> s)
+        return x
+    inv1, inv2 = pow(0xBF58476D1CE4E5B9, -1, 1 << 64), pow(0x94D049BB133111EB, -1, 1 << 64)
+    out = []
+    for v in values:
+        z = unshift(int(v), 31)
+        z = (z * inv2) & M
+        z = unshift(z, 27)
+        z = (z * inv1) & M
+        z = unshift(z, 30)
+        out.append(((z - 0x9E3779B97F4A7C15) & M) ^ seed)
+    return np.array(out, dtype=np.uint64)
+
+
+@pytest.mark.parametrize("rows", [1, 2, 3, 10, 100_000, 50_000_000, 10**9, 2**31, 2**32 - 1, 2**32, 2**32 + 1, 3 * 2**40 + 7,
+                                  2**62, 2**62 + 1, 2**63 - 1])
+def test_hash_modulo_at_chosen_hash_values(rows):
+    """The exact modulo on the values where a reciprocal-based remainder can go wrong: hash values at
+    and around multiples of `rows`, at the top of the 64-bit range, and around 2^32 and 2^63. The IDs
+    are constructed so that their hash IS the chosen value (checked through the oracle's own hash)."""
+    m = mfet()
+    seed = 0x243F6A8885A308D3
+    M64 = 1 << 64
+    want_h = {0, 1, rows - 1, rows, rows + 1, 2 * rows - 1, 2 * rows, M64 - 1, M64 - 2, M64 - rows, (M64 - 1) // rows * rows,
+              (M64 - 1) // rows * rows - 1, (M64 - 1) // rows * rows + rows - 1, 2**32 - 1, 2**32, 2**63 - 1, 2**63, 2**63 + 1}
+    rng = np.random.default_rng(rows % 977)
+    for _ in range(3000):  # multiples of rows, plus and minus one, all over the range
+        q = int(rng.integers(0, M64 // rows, dtype=np.uint64)) if rows < M64 // 2 else int(rng.integers(0, 2))
+        want_h.update({q * rows - 1, q * rows, q * rows + 1, q * rows + rows - 1})
+    hs = sorted(v for v in want_h if 0 <= v < M64)
+    ids = _ids_that_hash_to(hs, seed)
+    assert [orc.splitmix64(int(i) ^ seed) for i in ids[:50]] == hs[:50]  # the construction, against the oracle's hash
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    h = m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), rows, 4, m.F32, m.LOC_DEVICE, 0, seed, 0)])
+    try:
+        d_ids = torch.from_numpy(ids.view(np.int64)).cuda()
+        d_rows = torch.empty(ids.size, dtype=torch.int64, device="cuda")
+        m.mfet_hash_ids(h, 0, d_ids, ids.size, d_rows, _stream())
+        got = d_rows.cpu().numpy()
+        assert np.array_equal(got, orc.hash_ids(ids, seed, rows))
+        assert np.array_equal(got, np.array([v % rows for v in hs], dtype=np.int64))  # and against the plain definition
+    finally:
+        m.mfet_tables_destroy(h)
+
+
 @pytest.mark.parametrize("n", [1, 2, 3, 511, 513, 100_000, 100_001])
 @pytest.mark.parametrize("shift_in,shift_out", [(0, 0), (1, 0), (0, 1), (1, 1)])
 def test_hash_ids_any_length_and_alignment(n, shift_in, shift_out):
