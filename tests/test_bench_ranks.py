@@ -51,3 +51,31 @@ def test_single_process_aggregation_is_identity():
     batch = gi.make_batch(w, 0)
     nnz = int(batch.offsets[-1])
     assert b(w, batch) == nnz * 128 + nnz * 8 + (512 + 1) * 8 + 512 * 32 * 4
+
+
+def test_bench_bookkeeping_helpers(tmp_path, monkeypatch):
+    """Percentiles, row-lookup counts and the reading of the committed DRAM-traffic file (keyed by workload
+    and by a fingerprint of the kernel sources: a stale figure must come back as None)."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2508_05700_b200 import inputs as gi
+    s = bench.stats([1.0, 2.0, 3.0, 4.0, 100.0])
+    assert s["median"] == 3.0 and s["n"] == 5 and s["p10"] < s["median"] < s["p90"]
+    w = gi.make_workload(3, rows_scale=1e-4, batch_scale=1 / 64)
+    b = gi.make_batch(w, 0)
+    nnz = int(b.offsets[-1])
+    assert bench.row_lookups(w, b) == 3 * nnz                      # three facet slots read every feature's IDs
+    assert bench.row_lookups(w, b, [0]) == int(b.offsets[w.batch] - b.offsets[0])
+    t = w.tables
+    rows_bytes = sum(int(b.offsets[(f + 1) * w.batch] - b.offsets[f * w.batch]) * (t[3 * f].dim + t[3 * f + 1].dim + t[3 * f + 2].dim) * 2
+                     for f in range(w.n_features))
+    assert bench.algorithmic_bytes(w, b) == rows_bytes + nnz * 12 + (w.n_features * w.batch + 1) * 8 + w.batch * w.out_dim * 4
+    fp = bench.kernel_fingerprint()
+    prof = tmp_path / "profiles"
+    prof.mkdir()
+    (prof / "bag_kernel_dram_traffic.txt").write_text("# comment\nconfig3 %s 12345 scaled capture: x\nconfig2 deadbeefdeadbeef 777 old\n" % fp)
+    monkeypatch.setattr(bench, "ROOT", str(tmp_path))
+    monkeypatch.setattr(bench, "kernel_fingerprint", lambda: fp)
+    assert bench.recorded_traffic("config3") == (12345.0, "scaled capture: x")
+    assert bench.recorded_traffic("config2") == (None, None)       # captured for other kernel sources
+    assert bench.recorded_traffic("config9") == (None, None)
