@@ -69,8 +69,10 @@ enum {
                                    table in host memory and in mfet_embedding_bag_backward        */
   MFET_DEV_OFFSETS = 2u,        /* offsets decreased inside a bag; bag skipped */
   MFET_DEV_CAPACITY = 4u,       /* a host-path batch exceeded the workspace    */
-  MFET_DEV_BOUNDS = 8u          /* only in the bounds-checked build of the library: a kernel formed an
+  MFET_DEV_BOUNDS = 8u,         /* only in the bounds-checked build of the library: a kernel formed an
                                    index outside its array; the access was skipped               */
+  MFET_DEV_STALLED = 16u        /* a dedup tile waited two seconds for the counts of the tiles before
+                                   it and gave up: the dedup result of that call is undefined     */
 };
 
 /* One embedding table. Rows are `dim` elements of `dtype`, row-major.
@@ -255,7 +257,8 @@ MFET_API int mfet_cache_build(mfet_tables_t* t, int32_t table_id, const int64_t*
                      void* cache_mem, uint64_t cache_bytes, mfet_stream_t stream);
 
 /* Workspace for the host-table path and mfet_dedup_rows: device bytes needed to
- * handle up to `max_ids` IDs per host-table slot per call. */
+ * handle up to `max_ids` IDs per host-table slot per call; max_ids < 2^30 - 1
+ * (the dedup hands counts from tile to tile in 30 bits), else INVALID_ARG. */
 MFET_API int mfet_workspace_bytes(const mfet_tables_t* t, int64_t max_ids, uint64_t* bytes /*host*/);
 
 /* Attach a caller-owned, 256-byte-aligned device workspace sized by

@@ -291,7 +291,7 @@ int mfet_profile_read(mfet_tables_t* t, float* stage_ms) {
 }
 
 int mfet_workspace_bytes(const mfet_tables_t* t, int64_t max_ids, uint64_t* bytes) {
-  if (!t || !bytes || max_ids < 0) return MFET_ERR_INVALID_ARG;
+  if (!t || !bytes || max_ids < 0 || max_ids >= (1ll << 30) - 1) return MFET_ERR_INVALID_ARG;
   uint64_t max_row_bytes = 16;
   for (const TableHost& tb : t->tables)
     if (tb.desc.location == MFET_LOC_HOST && tb.row_bytes > max_row_bytes) max_row_bytes = tb.row_bytes;
@@ -300,7 +300,7 @@ int mfet_workspace_bytes(const mfet_tables_t* t, int64_t max_ids, uint64_t* byte
 }
 
 int mfet_set_workspace(mfet_tables_t* t, void* dev_ptr, uint64_t bytes, int64_t max_ids) {
-  if (!t || max_ids < 0) return MFET_ERR_INVALID_ARG;
+  if (!t || max_ids < 0 || max_ids >= (1ll << 30) - 1) return MFET_ERR_INVALID_ARG;
   if (!dev_ptr) {
     t->ws = nullptr;
     t->ws_bytes = 0;
@@ -313,11 +313,13 @@ int mfet_set_workspace(mfet_tables_t* t, void* dev_ptr, uint64_t bytes, int64_t 
   if (rc != MFET_OK) return rc;
   if (bytes < need) return MFET_ERR_WORKSPACE;
   {
-    // the arrival counters inside the workspace must start at zero (kernels leave them at zero)
+    // the dedup's digit totals inside the workspace must start at zero (its kernels leave them at zero)
     WsLayout L;
     workspace_layout(max_ids, 16, &L);
     DeviceGuard g(t->device);
-    if (!g.ok || cudaMemset(static_cast<uint8_t*>(dev_ptr) + L.counters, 0, 64) != cudaSuccess) return MFET_ERR_CUDA;
+    if (!g.ok || cudaMemset(static_cast<uint8_t*>(dev_ptr) + L.counters, 0, 64) != cudaSuccess ||
+        cudaMemset(static_cast<uint8_t*>(dev_ptr) + L.hist, 0, kDedupTotalsBytes) != cudaSuccess)
+      return MFET_ERR_CUDA;
   }
   t->ws = dev_ptr;
   t->ws_bytes = bytes;

@@ -30,7 +30,7 @@ OPT_OVERLAP_LAUNCHES = 5
 OK = 0
 ERR_INVALID_ARG, ERR_NOT_REGISTERED, ERR_ALIGNMENT, ERR_UNSUPPORTED_DIM = -1, -2, -3, -4
 ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -5, -6, -7
-DEV_ROW_RANGE, DEV_OFFSETS, DEV_CAPACITY, DEV_BOUNDS = 1, 2, 4, 8
+DEV_ROW_RANGE, DEV_OFFSETS, DEV_CAPACITY, DEV_BOUNDS, DEV_STALLED = 1, 2, 4, 8, 16
 
 EXPORTS = [
     "mfet_row_bytes", "mfet_tables_create", "mfet_tables_destroy", "mfet_host_tables_register",
