@@ -574,6 +574,45 @@ def test_dedup_bit_exact(n, hi):
         m.mfet_tables_destroy(h)
 
 
+def test_dedup_calls_of_changing_size_queued_on_one_workspace():
+    """Calls of very different sizes and key widths, queued back to back on one stream and one workspace
+    with no synchronisation in between: every call's kernels must find the tile counters, the digit
+    totals and the ping-pong buffers as the call before left them, wherever that call's tiles ended."""
+    m = mfet()
+    rng = np.random.default_rng(77)
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    h = m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), 8, 4, m.F32, m.LOC_DEVICE, 0, 0, 0)])
+    try:
+        cap = 700_000
+        ws = torch.empty(m.mfet_workspace_bytes(h, cap), dtype=torch.uint8, device="cuda")
+        m.mfet_set_workspace(h, ws, ws.numel(), cap)
+        calls = [(600_000, 10**9), (3, 5), (70_000, 2**40), (2048 * 16, 300), (2048 * 16 + 1, 10**6), (1, 1),
+                 (2048 * 17, 2**20), (650_000, 2**62), (4097, 256), (600_000, 10**9)]
+        held = []
+        for n, hi in calls:
+            rows = rng.integers(0, hi, size=n, dtype=np.int64)
+            if n > 100:
+                rows[rng.random(n) < 0.4] = rows[0]          # one very hot row
+            d_rows = torch.from_numpy(rows).cuda()
+            uniq = torch.full((n,), -7, dtype=torch.int64, device="cuda")
+            inv = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+            nu = torch.full((1,), -7, dtype=torch.int64, device="cuda")
+            held.append((rows, d_rows, uniq, inv, nu))
+        for _ in range(2):
+            for (n, hi), (rows, d_rows, uniq, inv, nu) in zip(calls, held):
+                m.mfet_dedup_rows(h, d_rows, n, uniq, inv, nu, hi, _stream())
+        torch.cuda.synchronize()
+        assert m.mfet_query_status(h) == 0
+        for (n, hi), (rows, d_rows, uniq, inv, nu) in zip(calls, held):
+            wu, wi = orc.dedup(rows)
+            k = int(nu.item())
+            assert k == wu.size, (n, hi)
+            assert np.array_equal(uniq.cpu().numpy()[:k], wu), (n, hi)
+            assert np.array_equal(inv.cpu().numpy(), wi), (n, hi)
+    finally:
+        m.mfet_tables_destroy(h)
+
+
 # -------------------------------------------------------------- host path ---
 
 def _hot_rows(dt, w, table_id, feature, count, rows_total):
