@@ -23,7 +23,8 @@ def build(force: bool = False, verbose: bool = False, checked: bool = False) -> 
     which every kernel tests its indices and reports a violation through MFET_DEV_BOUNDS."""
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     srcs = [os.path.join(CSRC, s) for s in SOURCES]
-    deps = srcs + [os.path.join(CSRC, "common.cuh"), os.path.join(HERE, "..", "include", "mfet.h")]
+    deps = srcs + [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "dedup_layout.cuh"),
+                   os.path.join(HERE, "..", "include", "mfet.h")]
     lib = LIB_CHECKED if checked else LIB
     if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _newest(deps):
         return lib

@@ -6,6 +6,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "dedup_layout.cuh"
 
 using namespace mfet;
 

@@ -196,10 +196,6 @@ struct CacheDev {
   uint32_t pad;
 };
 
-// The dedup's digit totals sit at the start of WsLayout::hist and must be zero between calls: the
-// library clears them when a workspace is set, and every call leaves them at zero.
-constexpr uint64_t kDedupTotalsBytes = 8 * 256 * 4;
-
 struct WsLayout {
   uint64_t keys_a, keys_b, idx_a, idx_b, hist, tile_counts, counters, uniq, inverse, src, miss_rows,
       staging, total;

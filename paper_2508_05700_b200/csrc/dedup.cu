@@ -11,6 +11,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "dedup_layout.cuh"
 
 namespace mfet {
 
