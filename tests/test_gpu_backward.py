@@ -61,11 +61,14 @@ def test_backward_matches_oracle(config, rows_scale, batch_scale):
 
 
 @pytest.mark.parametrize("B,max_len,rows,dim,pool", [(300, 40, 7, 136, 2), (300, 40, 1, 8, 1), (3, 4, 5, 264, 0),
-                                                    (64, 300, 3, 32, 0)])
+                                                    (64, 300, 3, 32, 0), (5000, 6, 2, 136, 1), (1025, 30, 3, 72, 2),
+                                                    (2048, 12, 40, 128, 0)])
 def test_backward_hot_rows_and_tiny_workspaces(B, max_len, rows, dim, pool):
     """A few rows that receive hundreds or thousands of lookups each (their runs are summed in pieces
-    by many warps and combined), more than 128 columns, and a workspace too small to hold partial
-    sums (then one warp sums everything): the sparse gradient against the oracle's dense scatter-add."""
+    by many warps and combined; runs of more than 32 pieces by a whole block), more than 128 columns,
+    column counts that are no multiple of 32, batches of more than 1024 samples (the bag search then
+    starts in an excerpt of the offsets) and a workspace too small to hold partial sums (then one warp
+    sums everything): the sparse gradient against the oracle's dense scatter-add."""
     m = mfet()
     rng = np.random.default_rng(B * 1000 + dim)
     spec = gi.TableSpec(rows, dim, gi.F32, 0x5EED, 0x1234)

@@ -574,6 +574,22 @@ def test_dedup_bit_exact(n, hi):
         m.mfet_tables_destroy(h)
 
 
+def test_workspace_capacity_limit():
+    """The dedup hands counts from tile to tile in 30 bits: a workspace for 2^30 - 1 IDs or more is refused
+    by name, before anything is launched."""
+    m = mfet()
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    h = m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), 8, 4, m.F32, m.LOC_DEVICE, 0, 0, 0)])
+    try:
+        assert m.mfet_workspace_bytes(h, (1 << 30) - 2) > 0
+        for bad in ((1 << 30) - 1, 1 << 30, 1 << 40):
+            with pytest.raises(m.MfetError) as e:
+                m.mfet_workspace_bytes(h, bad)
+            assert e.value.status == m.ERR_INVALID_ARG
+    finally:
+        m.mfet_tables_destroy(h)
+
+
 def test_dedup_calls_of_changing_size_queued_on_one_workspace():
     """Calls of very different sizes and key widths, queued back to back on one stream and one workspace
     with no synchronisation in between: every call's kernels must find the tile counters, the digit
