@@ -677,6 +677,30 @@ def test_host_table_path_matches_oracle_and_hbm_placement(pinned_by_caller):
     assert_close(hbm[:, :64], cold[:, :64])
 
 
+def test_host_table_feature_without_a_single_id():
+    """A batch in which the host-table feature has only empty bags: the sort runs over zero keys (the count
+    is read on the device), the slot's columns are zeros, nothing is fetched, no error bit is set, and the
+    batch after it finds the workspace's counters as a normal batch leaves them."""
+    w = gi.make_workload(5, rows_scale=0.001, batch_scale=0.0625)
+    b = gi.make_batch(w, 0)
+    B = w.batch
+    cut = int(b.offsets[B])                                   # the IDs of feature 0 (the host table's)
+    off = b.offsets.copy()
+    off[:B + 1] = 0
+    off[B + 1:] -= cut
+    hollow = gi.Batch(b.ids[cut:].copy(), off, None if b.weights is None else b.weights[cut:].copy())
+    with DeviceTables(w.tables) as dt:
+        dt.set_workspace(cut + 1024)
+        full_before = workload_forward(dt, w, b)
+        got = workload_forward(dt, w, hollow)
+        assert dt.m.mfet_query_status(dt.h) == 0
+        assert dt.m.mfet_host_path_counts(dt.h) == (0, 0)
+        assert not got[:, :w.tables[0].dim].any()
+        assert_close(got, workload_oracle(dt, w, hollow), "host-table feature with no IDs")
+        assert np.array_equal(workload_forward(dt, w, b), full_before)
+        assert dt.m.mfet_query_status(dt.h) == 0
+
+
 @pytest.mark.parametrize("cache_share", [0.0, 0.02, 1.0])
 def test_cache_probe_and_miss_list_against_a_host_computation(cache_share):
     """The host-table slot's intermediate results, read back: distinct rows = numpy's sorted unique
