@@ -3,10 +3,10 @@
 // same pass also probes the HBM hot-row cache and compacts the misses, so that
 // only distinct, uncached rows are fetched over PCIe.
 //
-// One launch counts the digits of all passes, one launch per 8-bit digit scatters, one launch
-// writes the unique rows and the inverse map. Inside a launch a tile learns the counts of the
-// tiles before it from status words in global memory (see below) instead of from a separate
-// scan launch. Results are canonical (ascending unique rows), hence bit-reproducible.
+// One launch counts the digits of all passes, one launch per 8-bit digit scatters, two launches
+// count and write the unique rows and the inverse map. Inside a scatter launch a tile learns the
+// counts of the tiles before it from status words in global memory (see below) instead of from a
+// separate scan launch. Results are canonical (ascending unique rows), hence bit-reproducible.
 #include <cstring>
 #include <mutex>
 
@@ -102,9 +102,9 @@ constexpr int kHistThreads = 1024;
 constexpr int kHistRounds = kSortTile / kHistThreads;
 
 // Digit counts of the whole input for every pass at once (the keys do not change from pass to
-// pass, only their order), added into total[pass][digit], which the caller has zeroed. With HASH
-// the keys are produced here from the raw IDs (a host-table slot) and stored for the passes.
-// Also clears the status words that the first pass and the unique kernel poll.
+// pass, only their order), added into total[pass][digit], which every call leaves at zero. With
+// HASH the keys are produced here from the raw IDs (a host-table slot) and stored for the passes.
+// Also clears the status words that the first pass polls and the group sums of the unique kernels.
 template <bool HASH>
 __global__ void __launch_bounds__(kHistThreads) digit_totals_kernel(NSrc ns, const uint64_t* __restrict__ keys_in,
                                                                     uint64_t* __restrict__ keys_store,
