@@ -574,6 +574,57 @@ def test_dedup_bit_exact(n, hi):
         m.mfet_tables_destroy(h)
 
 
+def test_dedup_on_two_streams_next_to_a_busy_pooling_stream():
+    """The sort's tiles wait for the counts of earlier tiles of the same launch. Two handles sort on two
+    streams while a third stream keeps the GPU's multiprocessors busy with pooling launches, so that tiles are
+    dispatched late and out of step: every result must still be exact and no wait may run out
+    (MFET_DEV_STALLED)."""
+    m = mfet()
+    rng = np.random.default_rng(5)
+    w = gi.make_workload(2, rows_scale=0.002, batch_scale=1.0)
+    b = gi.make_batch(w, 0)
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    hs = [m.mfet_tables_create([m.TableDesc(dummy.data_ptr(), 8, 4, m.F32, m.LOC_DEVICE, 0, 0, 0)]) for _ in range(2)]
+    try:
+        with DeviceTables(w.tables) as dt:
+            d_ids = torch.from_numpy(b.ids.view(np.int64)).cuda()
+            d_off = torch.from_numpy(b.offsets).cuda()
+            d_w = None if b.weights is None else torch.from_numpy(b.weights).cuda()
+            out = torch.empty(w.batch, w.out_dim, dtype=torch.float32, device="cuda")
+            shape, keep = m.make_shape(w.batch, w.n_features, w.slot_feature)
+            sizes = [(300_000, 10**9), (90_000, 5 * 10**7)]
+            work = []
+            for h, (n, hi) in zip(hs, sizes):
+                ws = torch.empty(m.mfet_workspace_bytes(h, n), dtype=torch.uint8, device="cuda")
+                m.mfet_set_workspace(h, ws, ws.numel(), n)
+                rows = rng.integers(0, hi, size=n, dtype=np.int64)
+                rows[rng.random(n) < 0.3] = rows[1]
+                work.append((ws, rows, torch.from_numpy(rows).cuda(), torch.empty(n, dtype=torch.int64, device="cuda"),
+                             torch.empty(n, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int64, device="cuda")))
+            torch.cuda.synchronize()
+            for it in range(150):
+                for _ in range(2):
+                    m.mfet_embedding_bag_forward(dt.h, shape, d_ids, d_off, d_w, w.table_ids, w.pooling, out,
+                                                 streams[2].cuda_stream)
+                for k, (h, (n, hi)) in enumerate(zip(hs, sizes)):
+                    ws, rows, d_rows, uniq, inv, nu = work[k]
+                    m.mfet_dedup_rows(h, d_rows, n, uniq, inv, nu, hi, streams[k].cuda_stream)
+            torch.cuda.synchronize()
+            for k, (h, (n, hi)) in enumerate(zip(hs, sizes)):
+                ws, rows, d_rows, uniq, inv, nu = work[k]
+                assert m.mfet_query_status(h) == 0
+                wu, wi = orc.dedup(rows)
+                kk = int(nu.item())
+                assert kk == wu.size
+                assert np.array_equal(uniq.cpu().numpy()[:kk], wu)
+                assert np.array_equal(inv.cpu().numpy(), wi)
+            assert m.mfet_query_status(dt.h) == 0
+    finally:
+        for h in hs:
+            m.mfet_tables_destroy(h)
+
+
 def test_workspace_capacity_limit():
     """The dedup hands counts from tile to tile in 30 bits: a workspace for 2^30 - 1 IDs or more is refused
     by name, before anything is launched."""
