@@ -70,8 +70,14 @@ __global__ void __launch_bounds__(256) cache_index_kernel(const int64_t* __restr
 cudaError_t launch_fetch(const uint8_t* table, uint64_t stride, uint32_t chunks, const int64_t* rows_list,
                          const int64_t* n_ptr, int64_t n_imm, uint8_t* dst, uint64_t table_rows, int64_t cap,
                          uint32_t* err, cudaStream_t s) {
-  fetch_rows_kernel<<<sm_count() * 4, 256, 0, s>>>(table, stride, chunks, rows_list, n_ptr, n_imm, dst, table_rows, cap,
-                                                   err);
+  // A small footprint on purpose: one warp per multiprocessor with kFetchUnroll loads per lane keeps about
+  // 2 400 rows in flight, far more than the host link needs (random rows arrive at 50-60 million a second,
+  // 2-3 us each). With 4 x 256 threads per multiprocessor (a) random rows came 20 % slower (6.2 instead of
+  // 7.8 GB/s on a 128 GB table: the hundreds of thousands of pending host reads get in one another's way),
+  // and (b) every other kernel that ran next to the fetch crawled behind them (a 20 us copy kernel took
+  // 1.1 ms; now 57 us) - and in the lookup path the pooling of one batch and the dedup of the next run
+  // next to it. Consecutive rows still arrive at 43 GB/s (48 with the large footprint).
+  fetch_rows_kernel<<<sm_count(), 32, 0, s>>>(table, stride, chunks, rows_list, n_ptr, n_imm, dst, table_rows, cap, err);
   return cudaGetLastError();
 }
 
